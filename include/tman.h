@@ -1,0 +1,131 @@
+/*
+ * tman.h -- C ABI of the low-bit-weight x fp16-activation matmul through table lookup
+ * (decode: bit-serial LUT mpGEMV; prefill: LUT dequantization fused into a tensor-core GEMM),
+ * written for NVIDIA B200 (sm_100a).
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *   - Nothing is allocated, nothing is kept between calls, the device is never synchronised
+ *     (except tman_read_status), all work is enqueued on `stream`.
+ *   - The return value is a tman_status.  Argument errors are reported before anything is
+ *     enqueued.  Errors only the device can see (a packed buffer whose header does not match
+ *     the arguments, a bounded wait that ran out) are written to the first 32-bit word of the
+ *     workspace ("status word"); read it with tman_read_status after the stream has drained.
+ *     A kernel that finds a bad header leaves its outputs untouched.
+ *   - Shapes: M tokens (rows of x), K input channels (reduction), N output channels.
+ *     W is logically [K x N]:  w[k][n] = s[k/group][n] * (q[k][n] - z[k/group][n])
+ *     (paper Sec. 2.2, "Dequantization-based low-bit inference"), q and z unsigned integers
+ *     in [0, 2^bits).
+ *   - Legal shapes: bits in {1,2,3,4} for pack/unpack, {2,3,4} for the matmuls;
+ *     group in {32,64,128}; K % 128 == 0; N % 8 == 0.  Anything else: TMAN_ERR_SHAPE /
+ *     TMAN_ERR_UNSUPPORTED.
+ */
+#ifndef TMAN_H_
+#define TMAN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Same type as the CUDA runtime's cudaStream_t (an opaque CUstream_st pointer). */
+typedef struct CUstream_st *tman_stream_t;
+
+typedef enum {
+    TMAN_OK = 0,
+    TMAN_ERR_NULL = 1,             /* a required pointer is NULL */
+    TMAN_ERR_SHAPE = 2,            /* K, N, M, bits or group outside the legal set */
+    TMAN_ERR_UNSUPPORTED = 3,      /* legal for the format, not for this call */
+    TMAN_ERR_BUFFER_TOO_SMALL = 4, /* packed buffer or workspace smaller than required */
+    TMAN_ERR_BAD_PACKED = 5,       /* (device-side) header does not match the arguments */
+    TMAN_ERR_CUDA = 6,             /* a CUDA runtime/driver call or a launch failed */
+    TMAN_ERR_TIMEOUT = 7           /* (device-side) a bounded wait ran out */
+} tman_status;
+
+/* Human-readable name of a status code (host pointer to a static string). */
+const char *tman_status_string(int status);
+
+/* Library version, 1000*major + minor. */
+int tman_version(void);
+
+/* ---- sizes (host only, no GPU touched) ------------------------------------------------ */
+
+/* Bytes of the packed weight buffer (256-byte header + bit-plane words + scales + zeros,
+ * each section padded to 256 bytes).  Paper Sec. 4.1: one bit-serial copy of the weights
+ * serves both decode and prefill. */
+tman_status tman_packed_bytes(int K, int N, int bits, int group, size_t *out_bytes /*host*/);
+
+/* Bytes of scratch a call needs.  op: 0 = tman_mpgemv, 1 = tman_mpgemm, 2 = unpack / debug
+ * extractors.  The workspace must have been cleared once with tman_workspace_init before its
+ * first use; calls leave it ready for the next call.  Two calls that overlap on the GPU must
+ * not share a workspace. */
+tman_status tman_workspace_bytes(int op, int M, int K, int N, int bits, int group,
+                                 size_t *out_bytes /*host*/);
+
+/* Zero a workspace (status word and split-K arrival counters). */
+tman_status tman_workspace_init(void *workspace, size_t ws_bytes, tman_stream_t stream);
+
+/* Copy the workspace's status word to *out_status (host) and wait for `stream`. */
+tman_status tman_read_status(const void *workspace, int *out_status /*host*/,
+                             tman_stream_t stream);
+
+/* ---- offline repack (paper Sec. 4.1 "Unified Layout", Sec. 2.2 bit-serial decomposition) -- */
+
+/* codes  uint8 [K][N], one code per byte, values in [0, 2^bits)
+ * scales fp16  [K/group][N]
+ * zeros  uint8 [K/group][N], values in [0, 2^bits)
+ * packed: output, packed_bytes >= tman_packed_bytes(...), 256-byte aligned.
+ * Layout written (little endian):
+ *   header (256 B): "TMANB200", u32 version=1, u32 K, N, bits, group, lut_g=4,
+ *                   u64 planes_off, scales_off, zeros_off, total_bytes
+ *   planes: u32 word[((nb*bits + i)*(K/32) + v)*4 + c], n = 4*nb + c; bit r of the word is
+ *           bit i of q[32*v + r][n].  Nibble e of the word is the paper's 4-bit table index
+ *           of plane i for activations 32v+4e .. 32v+4e+3.
+ *   scales: fp16 [((nb*(K/group) + B)*4 + c]
+ *   zeros : u16  [nb*(K/group) + B], nibble c = z[B][4*nb + c]                              */
+tman_status tman_pack_weights(const uint8_t *codes, const void *scales_f16, const uint8_t *zeros,
+                              int K, int N, int bits, int group,
+                              void *packed, size_t packed_bytes, tman_stream_t stream);
+
+/* Inverse of tman_pack_weights (for round-trip checks).  Header mismatch -> status word. */
+tman_status tman_unpack_weights(const void *packed, size_t packed_bytes,
+                                int K, int N, int bits, int group,
+                                uint8_t *codes, void *scales_f16, uint8_t *zeros,
+                                void *workspace, size_t ws_bytes, tman_stream_t stream);
+
+/* ---- the two matmuls:  y[M][N] (fp16, row-major) = x[M][K] (fp16, row-major) . W ---------- */
+
+/* Decode (paper Sec. 2.2 "Bit-serial table lookup", Fig. 2; Sec. 4.3): activation tables are
+ * built in shared memory, packed bit-plane bytes index them, partial sums are
+ * shift-accumulated per quantization block, scaled, and summed across blocks in fp32.
+ * M in [1, 8]. */
+tman_status tman_mpgemv(const void *packed, const void *x_f16, void *y_f16,
+                        int M, int K, int N, int bits, int group,
+                        void *workspace, size_t ws_bytes, tman_stream_t stream);
+
+/* Prefill (paper Sec. 4.1 two-level LUT dequantization, Fig. 7; Sec. 4.2 three-stage pipeline,
+ * Fig. 9): packed tiles are staged in shared memory, rebuilt into fp16 tiles through the
+ * repack step and the per-(block, column) conversion table, and multiplied on the tensor
+ * cores with fp32 accumulation.  M >= 1. */
+tman_status tman_mpgemm(const void *packed, const void *x_f16, void *y_f16,
+                        int M, int K, int N, int bits, int group,
+                        void *workspace, size_t ws_bytes, tman_stream_t stream);
+
+/* ---- test-only extractors of the integer / table intermediates -------------------------- */
+
+/* idx uint8 [bits][K/4][N]: the 4-bit table index of every (plane, 4 activations, column)
+ * as the kernels read it out of the packed buffer (paper Sec. 4.1 "4-bit LUT index"). */
+tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int group,
+                               uint8_t *idx, void *workspace, size_t ws_bytes,
+                               tman_stream_t stream);
+
+/* lut fp32 [M][K/4][16]: lut[m][t][p] = sum_{j<4} x[m][4t+j] * bit_j(p), computed by the same
+ * device routine the decode kernel builds its tables from (paper Sec. 2.2). */
+tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TMAN_H_ */

@@ -1,0 +1,145 @@
+"""ctypes binding of libtman.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors (PyTorch supplies device memory and streams); every step of the
+path runs in the library's kernels.  There is no CPU fallback: if the shared library is missing
+the import of any entry point raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libtman.so")
+
+TMAN_OK = 0
+STATUS_NAMES = {
+    0: "TMAN_OK", 1: "TMAN_ERR_NULL", 2: "TMAN_ERR_SHAPE", 3: "TMAN_ERR_UNSUPPORTED",
+    4: "TMAN_ERR_BUFFER_TOO_SMALL", 5: "TMAN_ERR_BAD_PACKED", 6: "TMAN_ERR_CUDA", 7: "TMAN_ERR_TIMEOUT",
+}
+OP_GEMV, OP_GEMM, OP_AUX = 0, 1, 2
+
+EXPORTS = [
+    "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
+    "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
+    "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts",
+]
+
+_lib = None
+
+
+class TmanError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+        self.status = status
+
+
+def lib() -> C.CDLL:
+    """Load libtman.so (built by paper_2511_11248_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2511_11248_b200.build`; "
+                "there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        L.tman_status_string.restype = C.c_char_p
+        L.tman_status_string.argtypes = [C.c_int]
+        L.tman_version.restype = C.c_int
+        i, sz, vp = C.c_int, C.c_size_t, C.c_void_p
+        L.tman_packed_bytes.argtypes = [i, i, i, i, C.POINTER(sz)]
+        L.tman_workspace_bytes.argtypes = [i, i, i, i, i, i, C.POINTER(sz)]
+        L.tman_workspace_init.argtypes = [vp, sz, vp]
+        L.tman_read_status.argtypes = [vp, C.POINTER(i), vp]
+        L.tman_pack_weights.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
+        L.tman_unpack_weights.argtypes = [vp, sz, i, i, i, i, vp, vp, vp, vp, sz, vp]
+        L.tman_mpgemv.argtypes = [vp, vp, vp, i, i, i, i, i, vp, sz, vp]
+        L.tman_mpgemm.argtypes = [vp, vp, vp, i, i, i, i, i, vp, sz, vp]
+        L.tman_debug_indices.argtypes = [vp, i, i, i, i, vp, vp, sz, vp]
+        L.tman_debug_luts.argtypes = [vp, i, i, vp, vp]
+        for name in EXPORTS[2:]:
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(st: int, where: str) -> None:
+    if st != TMAN_OK:
+        raise TmanError(st, where)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _stream(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def tman_version() -> int:
+    return int(lib().tman_version())
+
+
+def tman_status_string(status: int) -> str:
+    return lib().tman_status_string(int(status)).decode()
+
+
+def tman_packed_bytes(K: int, N: int, bits: int, group: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib().tman_packed_bytes(K, N, bits, group, C.byref(out)), "tman_packed_bytes")
+    return int(out.value)
+
+
+def tman_workspace_bytes(op: int, M: int, K: int, N: int, bits: int, group: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib().tman_workspace_bytes(op, M, K, N, bits, group, C.byref(out)), "tman_workspace_bytes")
+    return int(out.value)
+
+
+def tman_workspace_init(workspace, stream=None) -> None:
+    _check(lib().tman_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                     _stream(stream)), "tman_workspace_init")
+
+
+def tman_read_status(workspace, stream=None) -> int:
+    out = C.c_int(0)
+    _check(lib().tman_read_status(_ptr(workspace), C.byref(out), _stream(stream)), "tman_read_status")
+    return int(out.value)
+
+
+def tman_pack_weights(codes, scales, zeros, K, N, bits, group, packed, stream=None) -> None:
+    _check(lib().tman_pack_weights(_ptr(codes), _ptr(scales), _ptr(zeros), K, N, bits, group,
+                                   _ptr(packed), packed.numel() * packed.element_size(),
+                                   _stream(stream)), "tman_pack_weights")
+
+
+def tman_unpack_weights(packed, K, N, bits, group, codes, scales, zeros, workspace, stream=None) -> None:
+    _check(lib().tman_unpack_weights(_ptr(packed), packed.numel() * packed.element_size(), K, N, bits,
+                                     group, _ptr(codes), _ptr(scales), _ptr(zeros), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream)),
+           "tman_unpack_weights")
+
+
+def tman_mpgemv(packed, x, y, M, K, N, bits, group, workspace, stream=None) -> None:
+    _check(lib().tman_mpgemv(_ptr(packed), _ptr(x), _ptr(y), M, K, N, bits, group, _ptr(workspace),
+                             workspace.numel() * workspace.element_size(), _stream(stream)),
+           "tman_mpgemv")
+
+
+def tman_mpgemm(packed, x, y, M, K, N, bits, group, workspace, stream=None) -> None:
+    _check(lib().tman_mpgemm(_ptr(packed), _ptr(x), _ptr(y), M, K, N, bits, group, _ptr(workspace),
+                             workspace.numel() * workspace.element_size(), _stream(stream)),
+           "tman_mpgemm")
+
+
+def tman_debug_indices(packed, K, N, bits, group, idx, workspace, stream=None) -> None:
+    _check(lib().tman_debug_indices(_ptr(packed), K, N, bits, group, _ptr(idx), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream(stream)),
+           "tman_debug_indices")
+
+
+def tman_debug_luts(x, M, K, lut, stream=None) -> None:
+    _check(lib().tman_debug_luts(_ptr(x), M, K, _ptr(lut), _stream(stream)), "tman_debug_luts")

@@ -1,0 +1,154 @@
+// C ABI: argument validation and dispatch.  No allocation, no global state, no device sync
+// (except tman_read_status, whose job is to wait).
+#include "common.cuh"
+
+using namespace tman;
+
+extern "C" {
+
+const char *tman_status_string(int status)
+{
+    switch (status) {
+        case TMAN_OK: return "TMAN_OK";
+        case TMAN_ERR_NULL: return "TMAN_ERR_NULL";
+        case TMAN_ERR_SHAPE: return "TMAN_ERR_SHAPE";
+        case TMAN_ERR_UNSUPPORTED: return "TMAN_ERR_UNSUPPORTED";
+        case TMAN_ERR_BUFFER_TOO_SMALL: return "TMAN_ERR_BUFFER_TOO_SMALL";
+        case TMAN_ERR_BAD_PACKED: return "TMAN_ERR_BAD_PACKED";
+        case TMAN_ERR_CUDA: return "TMAN_ERR_CUDA";
+        case TMAN_ERR_TIMEOUT: return "TMAN_ERR_TIMEOUT";
+        default: return "TMAN_ERR_UNKNOWN";
+    }
+}
+
+int tman_version(void) { return 1000 * 0 + 1; }
+
+tman_status tman_packed_bytes(int K, int N, int bits, int group, size_t *out_bytes)
+{
+    if (!out_bytes) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    *out_bytes = make_layout(K, N, bits, group).total;
+    return TMAN_OK;
+}
+
+tman_status tman_workspace_bytes(int op, int M, int K, int N, int bits, int group, size_t *out_bytes)
+{
+    if (!out_bytes) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    if (M < 1) return TMAN_ERR_SHAPE;
+    if (op == 0) {
+        if (M > 8) return TMAN_ERR_SHAPE;
+        *out_bytes = mpgemv_workspace_bytes(M, K, N);
+    } else if (op == 1) {
+        *out_bytes = mpgemm_workspace_bytes(M, K, N);
+    } else if (op == 2) {
+        *out_bytes = kWsStatusBytes;
+    } else {
+        return TMAN_ERR_UNSUPPORTED;
+    }
+    return TMAN_OK;
+}
+
+tman_status tman_workspace_init(void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    if (!workspace) return TMAN_ERR_NULL;
+    if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (cudaMemsetAsync(workspace, 0, ws_bytes, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return TMAN_ERR_CUDA;
+    return TMAN_OK;
+}
+
+tman_status tman_read_status(const void *workspace, int *out_status, tman_stream_t stream)
+{
+    if (!workspace || !out_status) return TMAN_ERR_NULL;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    uint32_t v = 0;
+    if (cudaMemcpyAsync(&v, workspace, sizeof(v), cudaMemcpyDeviceToHost, s) != cudaSuccess) return TMAN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return TMAN_ERR_CUDA;
+    *out_status = (int)v;
+    return TMAN_OK;
+}
+
+tman_status tman_pack_weights(const uint8_t *codes, const void *scales_f16, const uint8_t *zeros,
+                              int K, int N, int bits, int group,
+                              void *packed, size_t packed_bytes, tman_stream_t stream)
+{
+    if (!codes || !scales_f16 || !zeros || !packed) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    if (packed_bytes < make_layout(K, N, bits, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(packed) & 255) return TMAN_ERR_SHAPE;
+    return launch_pack(codes, scales_f16, zeros, K, N, bits, group, packed, reinterpret_cast<cudaStream_t>(stream));
+}
+
+tman_status tman_unpack_weights(const void *packed, size_t packed_bytes,
+                                int K, int N, int bits, int group,
+                                uint8_t *codes, void *scales_f16, uint8_t *zeros,
+                                void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    if (!codes || !scales_f16 || !zeros || !packed || !workspace) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    if (packed_bytes < make_layout(K, N, bits, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_unpack(packed, K, N, bits, group, codes, scales_f16, zeros,
+                         static_cast<uint32_t *>(workspace), reinterpret_cast<cudaStream_t>(stream));
+}
+
+static tman_status check_matmul(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
+                                int group, void *ws)
+{
+    if (!packed || !x || !y || !ws) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    if (bits < 2) return TMAN_ERR_UNSUPPORTED;
+    if (M < 1) return TMAN_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(packed) & 255) return TMAN_ERR_SHAPE;
+    return TMAN_OK;
+}
+
+tman_status tman_mpgemv(const void *packed, const void *x_f16, void *y_f16,
+                        int M, int K, int N, int bits, int group,
+                        void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    tman_status st = check_matmul(packed, x_f16, y_f16, M, K, N, bits, group, workspace);
+    if (st != TMAN_OK) return st;
+    if (M > 8) return TMAN_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(x_f16) & 15) return TMAN_ERR_SHAPE;
+    if (ws_bytes < mpgemv_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_mpgemv(packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
+                         reinterpret_cast<cudaStream_t>(stream));
+}
+
+tman_status tman_mpgemm(const void *packed, const void *x_f16, void *y_f16,
+                        int M, int K, int N, int bits, int group,
+                        void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    tman_status st = check_matmul(packed, x_f16, y_f16, M, K, N, bits, group, workspace);
+    if (st != TMAN_OK) return st;
+    if (ws_bytes < mpgemm_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_mpgemm(packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
+                         reinterpret_cast<cudaStream_t>(stream));
+}
+
+tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int group,
+                               uint8_t *idx, void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    if (!packed || !idx || !workspace) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_debug_indices(packed, K, N, bits, group, idx, static_cast<uint32_t *>(workspace),
+                                reinterpret_cast<cudaStream_t>(stream));
+}
+
+tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_stream_t stream)
+{
+    if (!x_f16 || !lut) return TMAN_ERR_NULL;
+    if (M < 1 || K < 4 || K % 4 != 0) return TMAN_ERR_SHAPE;
+    return launch_debug_luts(x_f16, M, K, lut, reinterpret_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

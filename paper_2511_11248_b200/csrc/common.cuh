@@ -1,0 +1,121 @@
+// Shared declarations of the CUDA side: packed-buffer layout, workspace layout, argument checks.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "tman.h"
+
+namespace tman {
+
+// ---- packed buffer -----------------------------------------------------------------------
+// 256-byte header, then bit-plane words, scales, zero-points (each section 256-byte padded).
+struct PackedHeader {
+    char     magic[8];      // "TMANB200"
+    uint32_t version;       // 1
+    uint32_t K, N, bits, group, lut_g;
+    uint64_t planes_off, scales_off, zeros_off, total_bytes;
+};
+static_assert(sizeof(PackedHeader) == 64, "header fields occupy the first 64 bytes");
+
+constexpr size_t   kHeaderBytes = 256;
+constexpr uint32_t kVersion = 1;
+
+__host__ __device__ inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+struct Layout {
+    size_t planes_off, scales_off, zeros_off, total;
+    size_t planes_bytes, scales_bytes, zeros_bytes;
+};
+
+__host__ __device__ inline Layout make_layout(int K, int N, int bits, int group)
+{
+    Layout L;
+    L.planes_bytes = (size_t)K * N * bits / 8;
+    L.scales_bytes = (size_t)(K / group) * N * 2;
+    L.zeros_bytes = (size_t)(K / group) * (N / 4) * 2;
+    L.planes_off = kHeaderBytes;
+    L.scales_off = L.planes_off + up256(L.planes_bytes);
+    L.zeros_off = L.scales_off + up256(L.scales_bytes);
+    L.total = L.zeros_off + up256(L.zeros_bytes);
+    return L;
+}
+
+// device-side header check: every kernel that reads a packed buffer calls it first
+__device__ inline bool header_matches(const void *packed, int K, int N, int bits, int group)
+{
+    const uint32_t *h = reinterpret_cast<const uint32_t *>(packed);
+    // "TMAN" = 0x4E414D54, "B200" = 0x30303242 (little endian)
+    bool ok = (h[0] == 0x4E414D54u) && (h[1] == 0x30303242u) && (h[2] == kVersion) &&
+              (h[3] == (uint32_t)K) && (h[4] == (uint32_t)N) && (h[5] == (uint32_t)bits) &&
+              (h[6] == (uint32_t)group) && (h[7] == 4u);
+    return ok;
+}
+
+// ---- workspace ---------------------------------------------------------------------------
+// [0, 256)              status word (u32) + padding
+// [256, 256 + ctr)      split-K arrival counters (u32), zero between calls
+// [256 + ctr, ...)      fp32 split-K partial sums
+constexpr size_t kWsStatusBytes = 256;
+
+__host__ __device__ inline size_t ws_counter_bytes(int N) { return up256((size_t)(N / 4) * 4); }
+
+// ---- argument checks (host) --------------------------------------------------------------
+inline tman_status check_format(int K, int N, int bits, int group)
+{
+    if (K <= 0 || N <= 0) return TMAN_ERR_SHAPE;
+    if (bits < 1 || bits > 4) return TMAN_ERR_SHAPE;
+    if (group != 32 && group != 64 && group != 128) return TMAN_ERR_SHAPE;
+    if (K % 128 != 0 || N % 8 != 0) return TMAN_ERR_SHAPE;
+    return TMAN_OK;
+}
+
+inline tman_status launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? TMAN_OK : TMAN_ERR_CUDA;
+}
+
+// number of SMs of the current device (queried per call; cheap attribute read)
+inline int sm_count()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return n;
+}
+
+// ---- table building block (device) -------------------------------------------------------
+// The 16 partial sums of four activations: out[p] = sum_{j<4} x_j * bit_j(p), accumulated in
+// increasing j (paper Sec. 2.2: each bit pattern indexes a precomputed sum).
+__device__ __forceinline__ void lut16(float x0, float x1, float x2, float x3, float (&out)[16])
+{
+    out[0] = 0.f;
+    out[1] = x0;
+    out[2] = x1;
+    out[3] = x0 + x1;
+    out[4] = x2;
+    out[5] = x0 + x2;
+    out[6] = x1 + x2;
+    out[7] = out[3] + x2;
+#pragma unroll
+    for (int p = 0; p < 8; ++p) out[8 + p] = (p == 0) ? x3 : out[p] + x3;
+}
+
+// entry points implemented per file
+tman_status launch_pack(const uint8_t *codes, const void *scales, const uint8_t *zeros, int K, int N,
+                        int bits, int group, void *packed, cudaStream_t s);
+tman_status launch_unpack(const void *packed, int K, int N, int bits, int group, uint8_t *codes,
+                          void *scales, uint8_t *zeros, uint32_t *status, cudaStream_t s);
+tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int group, uint8_t *idx,
+                                 uint32_t *status, cudaStream_t s);
+tman_status launch_debug_luts(const void *x, int M, int K, float *lut, cudaStream_t s);
+size_t      mpgemv_workspace_bytes(int M, int K, int N);
+tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
+                          int group, void *ws, size_t ws_bytes, cudaStream_t s);
+size_t      mpgemm_workspace_bytes(int M, int K, int N);
+tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
+                          int group, void *ws, size_t ws_bytes, cudaStream_t s);
+
+}  // namespace tman

@@ -1,0 +1,479 @@
+// Prefill path: two-level lookup dequantization fused into a tcgen05 GEMM
+// (paper Sec. 4.1 "Unified Layout through Fused LUT-based Dequantization", Fig. 7;
+//  Sec. 4.2 "Pipelining to Hide Dequantization Overhead", Fig. 9).
+//
+// One CTA computes a 128 x 128 tile of y.  Three kinds of agents run concurrently on a ring of
+// shared-memory stages guarded by mbarriers (the paper's DMA / vector-core / matrix-core stages):
+//   * warp 0, one lane : TMA loads of the fp16 activation tile (128 x 64, 128-byte swizzle);
+//   * warps 2..9       : read the packed bit-plane words of their column, rebuild the codes
+//                        (level 1: bit-serial -> bit-parallel), look every code up in the
+//                        per-(block, column) conversion table kept in registers and addressed
+//                        with byte-permute instructions (level 2: scale and zero-point baked in),
+//                        and write the fp16 weight tile in the K-major swizzled layout the
+//                        tensor core reads;
+//   * warp 1, one lane : tcgen05.mma (M128 N128 K16, fp16 x fp16 -> fp32 in tensor memory);
+//                        tcgen05.commit hands the stage back.
+// The dequantization warps then become the epilogue: tcgen05.ld, round to fp16, store.
+// Every wait is bounded: when a bound is hit the kernel records TMAN_ERR_TIMEOUT, stops issuing
+// work, and still reaches the common tear-down that frees tensor memory.
+#include "common.cuh"
+
+#include <cuda.h>
+
+namespace tman {
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 64;
+constexpr int NSTAGE = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int NUM_DEQ_WARPS = 8;
+constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS);
+constexpr int TMEM_COLS = 128;
+constexpr int SMEM_BYTES = NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+
+struct GemmParams {
+    const uint8_t  *packed;
+    const uint32_t *planes;
+    const __half   *scales;
+    const uint16_t *zeros;
+    __half         *y;
+    uint32_t       *status;
+    int M, K, N, bits, group;
+    int tiles_m, tiles_n;
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after about one second.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 1023u) == 1023u) {
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 1000000000ull) return false;
+        }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tcgen05_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tcgen05_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 fp16) and
+// which is stored with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                              // leading byte offset (unused here)
+    d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset: 8 rows
+    d |= (uint64_t)1 << 46;                              // descriptor version for this architecture
+    d |= (uint64_t)2 << 61;                              // 128-byte swizzle
+    return d;
+}
+
+// Byte permute with the full 4-bit selectors (bit 3 of a selector replicates the sign bit of the
+// selected byte), which the __byte_perm intrinsic does not expose.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// ---- level 2: per-(block, column) conversion table in registers ------------------------------
+// Entry c holds fp16( s * (c - z) ) (paper Sec. 4.1: integer-to-float conversion with scale and
+// zero-point pre-applied, 2^bits entries per quantization block).  Low and high bytes of the
+// entries are kept in separate byte tables so that one byte-permute looks up four codes.
+template <int BITS>
+struct ConvTable {
+    static constexpr int NQ = (BITS == 4) ? 4 : ((BITS == 3) ? 2 : 1);
+    uint32_t lo[NQ], hi[NQ];
+
+    __device__ __forceinline__ void build(__half s, uint32_t z)
+    {
+        const float sf = __half2float(s);
+        const float nsz = -sf * (float)z;
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const __half2 e01 = __floats2half2_rn(fmaf(sf, (float)(4 * q + 0), nsz), fmaf(sf, (float)(4 * q + 1), nsz));
+            const __half2 e23 = __floats2half2_rn(fmaf(sf, (float)(4 * q + 2), nsz), fmaf(sf, (float)(4 * q + 3), nsz));
+            const uint32_t h01 = *reinterpret_cast<const uint32_t *>(&e01);
+            const uint32_t h23 = *reinterpret_cast<const uint32_t *>(&e23);
+            lo[q] = __byte_perm(h01, h23, 0x6420);
+            hi[q] = __byte_perm(h01, h23, 0x7531);
+        }
+    }
+
+    // sel: four codes in the four low nibbles.  Returns the four low bytes / high bytes.
+    __device__ __forceinline__ void lookup(uint32_t sel, uint32_t &lb, uint32_t &hb) const
+    {
+        if constexpr (BITS <= 2) {
+            lb = __byte_perm(lo[0], lo[0], sel);
+            hb = __byte_perm(hi[0], hi[0], sel);
+        } else if constexpr (BITS == 3) {
+            lb = __byte_perm(lo[0], lo[1], sel);
+            hb = __byte_perm(hi[0], hi[1], sel);
+        } else {
+            const uint32_t sel7 = sel & 0x7777u;
+            // byte mask: 0xFF where the code's top bit is set (sign-replicating selectors)
+            const uint32_t mask = prmt(sel, sel << 4, 0x9D8Cu);
+            const uint32_t la = __byte_perm(lo[0], lo[1], sel7), lc = __byte_perm(lo[2], lo[3], sel7);
+            const uint32_t ha = __byte_perm(hi[0], hi[1], sel7), hc = __byte_perm(hi[2], hi[3], sel7);
+            lb = (la & ~mask) | (lc & mask);
+            hb = (ha & ~mask) | (hc & mask);
+        }
+    }
+};
+
+// 32 weights of one column (one plane word per bit) -> 16 half2 in natural k order.
+template <int BITS>
+__device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const ConvTable<BITS> &T, uint32_t (&out)[16])
+{
+    // level 1 (bit repacking): X[ph] nibble j = code of weight 4j + ph
+    uint32_t X[4];
+#pragma unroll
+    for (int ph = 0; ph < 4; ++ph) {
+        uint32_t x = 0;
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) x |= ((w[i] >> ph) & 0x11111111u) << i;
+        X[ph] = x;
+    }
+    // level 2 (conversion table) and re-pairing into adjacent k
+    uint32_t A[4][2], Bv[4][2];
+#pragma unroll
+    for (int ph = 0; ph < 4; ++ph)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t lb, hb;
+            T.lookup(X[ph] >> (16 * h), lb, hb);
+            A[ph][h] = __byte_perm(lb, hb, 0x5140);    // weights k0, k0+4   (k0 = 16h + ph)
+            Bv[ph][h] = __byte_perm(lb, hb, 0x7362);   // weights k0+8, k0+12
+        }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            out[8 * h + q]     = __byte_perm(A[2 * q][h], A[2 * q + 1][h], 0x5410);
+            out[8 * h + 2 + q] = __byte_perm(A[2 * q][h], A[2 * q + 1][h], 0x7632);
+            out[8 * h + 4 + q] = __byte_perm(Bv[2 * q][h], Bv[2 * q + 1][h], 0x5410);
+            out[8 * h + 6 + q] = __byte_perm(Bv[2 * q][h], Bv[2 * q + 1][h], 0x7632);
+        }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
+        return;
+    }
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *a_tiles = smem;
+    uint8_t *b_tiles = smem + NSTAGE * A_STAGE_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES));
+    // bars[0..NSTAGE) full, [NSTAGE..2NSTAGE) empty, [2NSTAGE] accumulator ready
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * NSTAGE + 1);
+    uint32_t *fail_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile_m = blockIdx.x % p.tiles_m, tile_n = blockIdx.x / p.tiles_m;
+    const int num_kb = p.K / BK;
+
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + NSTAGE), accum_bar = smem_u32(bars + 2 * NSTAGE);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(full0 + 8 * s, 1 + NUM_DEQ_WARPS);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accum_bar, 1);
+        *fail_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tcgen05_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tcgen05_relinquish();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
+
+    bool ok = true;
+    if (warp == 0) {
+        // ---- stage 1: activation tiles by TMA ------------------------------------------------
+        if (lane == 0) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % NSTAGE;
+                const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
+                if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
+                mbar_expect_tx(full0 + 8 * s, A_STAGE_BYTES);
+                tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, tile_m * BM, full0 + 8 * s);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- stage 3: tensor-core MMA --------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % NSTAGE;
+                const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
+                if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES));
+                const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
+#pragma unroll
+                for (int j = 0; j < BK / 16; ++j)
+                    tcgen05_mma_f16(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc, (kb > 0 || j > 0) ? 1u : 0u);
+                tcgen05_commit(empty0 + 8 * s);
+            }
+            if (ok) tcgen05_commit(accum_bar);
+        }
+    } else {
+        // ---- stage 2: two-level lookup dequantization ----------------------------------------
+        const int wd = warp - 2;
+        const int n_local = (wd & 3) * 32 + lane;
+        const int v = wd >> 2;                         // which of the two plane words of a k-block
+        const int n = tile_n * BN + n_local;
+        const bool valid = n < p.N;
+        const int nb = n >> 2, c = n & 3;
+        const int words_total = p.K / 32;
+        const int nblk = p.K / p.group;
+        const uint32_t *wp = p.planes + ((size_t)nb * BITS * words_total) * 4 + c;
+        const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
+        const uint32_t xr = (uint32_t)(n_local & 7);
+
+        ConvTable<BITS> T;
+        int cur_B = -1;
+        uint32_t wnext[BITS];
+#pragma unroll
+        for (int i = 0; i < BITS; ++i)
+            wnext[i] = valid ? __ldg(wp + ((size_t)i * words_total + v) * 4) : 0u;
+
+        for (int kb = 0; kb < num_kb; ++kb) {
+            const int s = kb % NSTAGE;
+            const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
+            uint32_t w[BITS];
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) w[i] = wnext[i];
+            if (kb + 1 < num_kb) {
+#pragma unroll
+                for (int i = 0; i < BITS; ++i)
+                    wnext[i] = valid ? __ldg(wp + ((size_t)i * words_total + 2 * (kb + 1) + v) * 4) : 0u;
+            }
+            const int Bk = ((2 * kb + v) * 32) / p.group;
+            if (Bk != cur_B) {
+                cur_B = Bk;
+                __half sv = __float2half(0.f);
+                uint32_t zz = 0;
+                if (valid) {
+                    sv = __ldg(p.scales + ((size_t)nb * nblk + Bk) * 4 + c);
+                    zz = ((uint32_t)__ldg(p.zeros + (size_t)nb * nblk + Bk) >> (4 * c)) & 0xFu;
+                }
+                T.build(sv, zz);
+            }
+            uint32_t out[16];
+            dequant_word<BITS>(w, T, out);
+            if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
+            uint8_t *row = b_tiles + s * B_STAGE_BYTES + row_off;
+#pragma unroll
+            for (int cj = 0; cj < 4; ++cj) {
+                const uint32_t chunk = ((uint32_t)(4 * v + cj)) ^ xr;
+                *reinterpret_cast<uint4 *>(row + chunk * 16) =
+                    make_uint4(out[4 * cj], out[4 * cj + 1], out[4 * cj + 2], out[4 * cj + 3]);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full0 + 8 * s);
+        }
+
+        // ---- epilogue: tensor memory -> fp16 -> global ----------------------------------------
+        if (ok && !mbar_wait(accum_bar, 0u)) ok = false;
+        if (ok) {
+            tcgen05_fence_after();
+            const int quarter = warp & 3;                 // tensor-memory lanes this warp may read
+            const int col_half = wd >> 2;                 // columns [0,64) or [64,128)
+            const int m = tile_m * BM + quarter * 32 + lane;
+#pragma unroll 1
+            for (int cc = 0; cc < 2; ++cc) {
+                const int col = col_half * 64 + cc * 32;
+                uint32_t r[32];
+                tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, r);
+                tcgen05_wait_ld();
+                if (m < p.M) {
+                    __half *dst = p.y + (size_t)m * p.N + (size_t)tile_n * BN + col;
+#pragma unroll
+                    for (int g8 = 0; g8 < 4; ++g8) {
+                        if (tile_n * BN + col + 8 * g8 < p.N) {
+                            uint32_t h[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __half2 t = __floats2half2_rn(__uint_as_float(r[8 * g8 + 2 * e]),
+                                                                    __uint_as_float(r[8 * g8 + 2 * e + 1]));
+                                h[e] = *reinterpret_cast<const uint32_t *>(&t);
+                            }
+                            *reinterpret_cast<uint4 *>(dst + 8 * g8) = make_uint4(h[0], h[1], h[2], h[3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    if (!ok) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tcgen05_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+    if (q != cudaDriverEntryPointSuccess) return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
+template <int BITS>
+tman_status launch_bits(const CUtensorMap &tmap, const GemmParams &p, cudaStream_t s)
+{
+    auto kern = mpgemm_kernel<BITS>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+        return TMAN_ERR_CUDA;
+    kern<<<p.tiles_m * p.tiles_n, GEMM_THREADS, SMEM_BYTES, s>>>(tmap, p);
+    return launch_status();
+}
+
+}  // namespace
+
+size_t mpgemm_workspace_bytes(int, int, int) { return kWsStatusBytes; }
+
+tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
+                          int group, void *ws, size_t, cudaStream_t s)
+{
+    if ((reinterpret_cast<uintptr_t>(x) & 15) != 0 || (reinterpret_cast<uintptr_t>(y) & 15) != 0) return TMAN_ERR_SHAPE;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return TMAN_ERR_CUDA;
+    CUtensorMap tmap;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return TMAN_ERR_CUDA;
+
+    Layout L = make_layout(K, N, bits, group);
+    const uint8_t *pk = static_cast<const uint8_t *>(packed);
+    GemmParams p;
+    p.packed = pk;
+    p.planes = reinterpret_cast<const uint32_t *>(pk + L.planes_off);
+    p.scales = reinterpret_cast<const __half *>(pk + L.scales_off);
+    p.zeros = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
+    p.y = static_cast<__half *>(y);
+    p.status = static_cast<uint32_t *>(ws);
+    p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
+    p.tiles_m = (M + BM - 1) / BM;
+    p.tiles_n = (N + BN - 1) / BN;
+    if (bits == 2) return launch_bits<2>(tmap, p, s);
+    if (bits == 3) return launch_bits<3>(tmap, p, s);
+    return launch_bits<4>(tmap, p, s);
+}
+
+}  // namespace tman

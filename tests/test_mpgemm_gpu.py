@@ -1,0 +1,90 @@
+"""Parity of tman_mpgemm (prefill path) with the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tman_oracle as orc
+from paper_2511_11248_b200 import binding as B, helpers as H, synth
+
+pytestmark = pytest.mark.gpu
+TOL = 5e-3   # max|gpu - ref| / max|ref|
+
+
+def run_gemm(c):
+    dev = H.device_case(c)
+    packed = H.pack_case(c, dev)
+    ws = H.alloc_workspace(B.OP_GEMM, c.M, c.K, c.N, c.bits, c.group)
+    y = torch.full((c.M, c.N), float("nan"), dtype=torch.float16, device="cuda")
+    B.tman_mpgemm(packed, dev["x"], y, c.M, c.K, c.N, c.bits, c.group, ws)
+    assert B.tman_read_status(ws) == 0
+    return y
+
+
+def check_full(c):
+    got = H.to_f64(run_gemm(c))
+    assert np.all(np.isfinite(got)), c.name
+    ref = orc.mpgemm(c.x, c.codes, c.scales, c.zeros, c.group)
+    e = float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
+    assert e <= TOL, (c.name, e)
+
+
+def check_sampled(c, n_rows=24):
+    """Full-size case: every output must be finite; sampled rows are compared one by one."""
+    y = run_gemm(c)
+    assert bool(torch.isfinite(y).all()), c.name
+    rng = np.random.default_rng(c.seed)
+    rows = np.unique(np.concatenate([[0, c.M - 1, min(c.M - 1, 127), min(c.M - 1, 128)],
+                                     rng.integers(0, c.M, size=n_rows)]))
+    ref = orc.mpgemm_rows(c.x, c.codes, c.scales, c.zeros, c.group, rows)
+    got = H.to_f64(y[torch.from_numpy(rows).cuda()])
+    e = float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
+    assert e <= TOL, (c.name, e)
+
+
+SMALL = [
+    # (M, K, N, bits, group): one tile, ragged M and N tiles, several k-blocks, every bit width
+    (128, 128, 128, 4, 128), (128, 256, 128, 2, 64), (1, 256, 8, 4, 64), (100, 384, 136, 3, 128),
+    (300, 512, 264, 4, 32), (257, 1024, 72, 2, 128), (129, 640, 392, 3, 64), (512, 2048, 256, 4, 64),
+]
+
+
+@pytest.mark.parametrize("M,K,N,bits,G", SMALL)
+def test_small_cases(M, K, N, bits, G):
+    check_full(synth.small_case(M, K, N, bits, G, seed=M + K + N + bits, outliers=(bits == 4)))
+
+
+def test_integer_case_is_exact():
+    rng = np.random.default_rng(5)
+    c = synth.small_case(130, 512, 136, 3, 64, seed=31)
+    c.x[:] = rng.integers(-2, 3, size=c.x.shape).astype(np.float16)
+    c.scales[:] = 1.0
+    c.zeros[:] = 0
+    got = H.to_f64(run_gemm(c))
+    want = c.x.astype(np.int64) @ c.codes.astype(np.int64)
+    assert np.array_equal(got, want.astype(np.float16).astype(np.float64))
+
+
+def test_gemm_and_gemv_read_the_same_packed_buffer():
+    c = synth.small_case(4, 1024, 264, 4, 64, seed=32)
+    dev = H.device_case(c)
+    packed = H.pack_case(c, dev)
+    wsv = H.alloc_workspace(B.OP_GEMV, c.M, c.K, c.N, c.bits, c.group)
+    wsm = H.alloc_workspace(B.OP_GEMM, c.M, c.K, c.N, c.bits, c.group)
+    yv = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
+    ym = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
+    B.tman_mpgemv(packed, dev["x"], yv, c.M, c.K, c.N, c.bits, c.group, wsv)
+    B.tman_mpgemm(packed, dev["x"], ym, c.M, c.K, c.N, c.bits, c.group, wsm)
+    ref = orc.mpgemm(c.x, c.codes, c.scales, c.zeros, c.group)
+    scale = np.max(np.abs(ref))
+    assert np.max(np.abs(H.to_f64(yv) - ref)) / scale <= TOL
+    assert np.max(np.abs(H.to_f64(ym) - ref)) / scale <= TOL
+
+
+@pytest.mark.parametrize("spec", synth.config4_specs(), ids=lambda s: s[0])
+def test_config4(spec):
+    check_sampled(synth.case_from_spec(spec), n_rows=48)
+
+
+@pytest.mark.parametrize("spec", synth.config5_specs(), ids=lambda s: s[0])
+def test_config5(spec):
+    check_sampled(synth.case_from_spec(spec, outliers=True), n_rows=12)

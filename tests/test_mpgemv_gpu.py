@@ -1,0 +1,101 @@
+"""Parity of tman_mpgemv (decode path) with the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tman_oracle as orc
+from paper_2511_11248_b200 import binding as B, helpers as H, synth
+
+pytestmark = pytest.mark.gpu
+TOL = 5e-3   # max|gpu - ref| / max|ref|, the bound the task states for fp32 accumulation
+
+
+def run_gemv(c, dev=None, packed=None):
+    dev = dev or H.device_case(c)
+    packed = packed if packed is not None else H.pack_case(c, dev)
+    ws = H.alloc_workspace(B.OP_GEMV, c.M, c.K, c.N, c.bits, c.group)
+    y = torch.full((c.M, c.N), float("nan"), dtype=torch.float16, device="cuda")
+    B.tman_mpgemv(packed, dev["x"], y, c.M, c.K, c.N, c.bits, c.group, ws)
+    assert B.tman_read_status(ws) == 0
+    return H.to_f64(y), ws, packed, dev
+
+
+def rel_err(got, ref):
+    assert np.all(np.isfinite(got))
+    return float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
+
+
+def check(c):
+    got, *_ = run_gemv(c)
+    ref = orc.mpgemm(c.x, c.codes, c.scales, c.zeros, c.group)
+    e = rel_err(got, ref)
+    assert e <= TOL, (c.name, e)
+    return e
+
+
+SMALL = [
+    # (M, K, N, bits, group): ragged K-slices (K not a multiple of 1024), ragged column units,
+    # single-slice K, every M, every bit width and group size
+    (1, 128, 8, 4, 128), (1, 1024, 32, 2, 64), (1, 1152, 40, 2, 32), (1, 2048, 264, 4, 64),
+    (1, 3584, 72, 3, 128), (2, 1024, 64, 2, 64), (2, 640, 24, 4, 32), (3, 2048, 136, 3, 64),
+    (4, 1280, 520, 4, 128), (5, 1024, 48, 2, 128), (6, 512, 8, 3, 32), (7, 2304, 200, 4, 64),
+    (8, 4096, 1032, 2, 64), (1, 18944, 16, 4, 128),
+]
+
+
+@pytest.mark.parametrize("M,K,N,bits,G", SMALL)
+def test_small_cases(M, K, N, bits, G):
+    check(synth.small_case(M, K, N, bits, G, seed=M * 1000 + bits * 10 + G))
+
+
+def test_repeat_calls_share_workspace_and_agree():
+    c = synth.small_case(2, 2048, 264, 4, 64, seed=21)
+    dev = H.device_case(c)
+    packed = H.pack_case(c, dev)
+    ws = H.alloc_workspace(B.OP_GEMV, c.M, c.K, c.N, c.bits, c.group)
+    ys = []
+    for _ in range(3):
+        y = torch.empty((c.M, c.N), dtype=torch.float16, device="cuda")
+        B.tman_mpgemv(packed, dev["x"], y, c.M, c.K, c.N, c.bits, c.group, ws)
+        ys.append(y)
+    assert B.tman_read_status(ws) == 0
+    assert torch.equal(ys[0], ys[1]) and torch.equal(ys[1], ys[2])   # fixed summation order
+
+
+def test_exact_special_cases():
+    # all-zero codes with z = 0 give exactly zero; codes == zero-point give (near) zero
+    c = synth.small_case(1, 2048, 64, 4, 64, seed=22)
+    c.codes[:] = 0
+    c.zeros[:] = 0
+    got, *_ = run_gemv(c)
+    assert np.all(got == 0.0)
+    # integers, unit scale, zero zero-point: exact (all sums are small integers)
+    rng = np.random.default_rng(3)
+    c = synth.small_case(2, 1024, 32, 3, 64, seed=23)
+    c.x[:] = rng.integers(-4, 5, size=c.x.shape).astype(np.float16)
+    c.scales[:] = 1.0
+    c.zeros[:] = 0
+    got, *_ = run_gemv(c)
+    want = c.x.astype(np.int64) @ c.codes.astype(np.int64)
+    assert np.array_equal(got, want.astype(np.float64))
+    # one-hot activation reads out single weights
+    c = synth.small_case(1, 1024, 32, 4, 64, seed=24)
+    c.x[:] = 0
+    c.x[0, 777] = 1.0
+    got, *_ = run_gemv(c)
+    want = c.scales.astype(np.float64)[777 // 64] * (c.codes[777].astype(np.float64) - c.zeros[777 // 64])
+    assert np.allclose(got[0], want.astype(np.float16).astype(np.float64), rtol=1e-3, atol=1e-6)
+
+
+def test_config1_full():
+    check(synth.config1())
+
+
+@pytest.mark.parametrize("spec", synth.config2_specs(), ids=lambda s: s[0])
+def test_config2_full(spec):
+    check(synth.case_from_spec(spec))
+
+
+@pytest.mark.parametrize("spec", synth.config3_specs(), ids=lambda s: s[0])
+def test_config3_full(spec):
+    check(synth.case_from_spec(spec))
