@@ -1,0 +1,412 @@
+#!/usr/bin/env python
+"""Benchmark of the table-lookup low-bit matmul path on B200.
+
+Headline (value): decode mpGEMV weight-stream GB/s on the 2-bit Llama-3-8B MLP shapes, M = 1
+(gate and up 4096 -> 14336, down 14336 -> 4096, group 64).  One step = the three mpGEMV calls
+of one MLP block over one token.  The packed weights rotate through several resident copies
+whose total size exceeds L2, so every call streams from HBM.  Steps are replayed from a CUDA
+graph and timed with CUDA events on the launching stream.
+
+Also reported on the same JSON line: the prefill mpGEMM rate (M = 1024, K = 4096,
+N in {4096, 14336}, 4-bit, group 128) with its tensor roofline; the end-to-end rate through the
+C ABI with host buffers; the CPU oracle's rate on a bounded sample; clocks sampled during the
+timed region.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (launched under torchrun) every rank runs an independent replica of the same step
+(the path does not shard); value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mpGEMV weight-stream GB/s (decode, 2-bit Llama-3-8B MLP, M=1)"
+UNIT = "GB/s"
+WORKLOAD = "config2: decode mpGEMV M=1, 2-bit, group 64, Llama-3-8B MLP gate/up 4096x14336 + down 14336x4096"
+MLP = [("gate", 4096, 14336), ("up", 4096, 14336), ("down", 14336, 4096)]
+BITS, GROUP = 2, 64
+NSETS = 6
+GRAPH_STEPS = 60
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_FP16_TFLOPS = 2250.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_TFLOPS = 1590.0
+
+
+def weight_bytes(K, N, bits, group):
+    """Algorithmic weight-stream bytes of one matrix: planes + fp16 scales + b-bit zero-points."""
+    return K * N * bits // 8 + (K // group) * N * 2 + (K // group) * N * bits // 8
+
+
+def total_bytes(M, K, N, bits, group):
+    return weight_bytes(K, N, bits, group) + M * K * 2 + M * N * 2
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm": float(d["hbm_gbs"]), "tf_burst": float(d["bf16_tflops"]),
+                "tf_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "src": "measured"}
+    return {"hbm": FALLBACK_HBM_GBS, "tf_burst": FALLBACK_TFLOPS, "tf_sustained": 1400.0, "src": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._t = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, nm in names.items():
+                    if r & bit:
+                        self.reasons.add(nm)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._t is not None:
+            self._t.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ---- reference arm: the CPU oracle, as it stands --------------------------------------------
+
+def oracle_step_sample(cases, n_cols):
+    """One oracle 'step' over the first n_cols output columns of each MLP matrix."""
+    from oracle import tman_oracle as orc
+    outs = []
+    for c in cases:
+        nc = min(n_cols, c.N)
+        outs.append(orc.mpgemm(c.x, np.ascontiguousarray(c.codes[:, :nc]),
+                               np.ascontiguousarray(c.scales[:, :nc]),
+                               np.ascontiguousarray(c.zeros[:, :nc]), c.group))
+    return outs
+
+
+def time_oracle(cases, n_cols, steps, warmup):
+    for _ in range(warmup):
+        oracle_step_sample(cases, n_cols)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step_sample(cases, n_cols)
+    dt = time.perf_counter() - t0
+    wb = sum(weight_bytes(c.K, min(n_cols, c.N), c.bits, c.group) for c in cases)
+    return dt / steps, wb
+
+
+def host_cases(seed_offset=0):
+    from paper_2511_11248_b200 import synth
+    lo, hi = synth.scale_range(BITS)
+    return [synth.make_case(f"c2_{nm}", 1, K, N, BITS, GROUP, synth.SEED_BASE + 200 + i + 10 * seed_offset, lo, hi)
+            for i, (nm, K, N) in enumerate(MLP)]
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import tman_oracle as orc
+    cases = host_cases()
+    # size the per-step sample so that the whole run stays within a couple of minutes
+    t_probe, _ = time_oracle(cases, 512, 1, 1)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    n_cols = int(max(8, min(14336, 512 * budget / max(t_probe, 1e-6)) // 8 * 8))
+    n_cols = min(n_cols, 14336)
+    sec, wb = time_oracle(cases, n_cols, args.steps, args.warmup)
+    val = wb / sec / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": f"first {n_cols} output columns of each matrix per step"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+                         "sample": f"first {n_cols} output columns of each of the 3 matrices, per step"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ---- our arm ---------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2511_11248_b200 import binding as B, helpers as H, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    B.lib()   # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    peaks = measured_peaks()
+    stream = torch.cuda.current_stream()
+
+    # ---- decode workload: NSETS resident weight sets (> L2 in total) ---------------------------
+    sets = []
+    host0 = None
+    for si in range(NSETS):
+        cases = host_cases(seed_offset=si)
+        if si == 0:
+            host0 = cases
+        entry = []
+        for c in cases:
+            dev = H.device_case(c)
+            packed = H.pack_case(c, dev)
+            y = torch.empty((1, c.N), dtype=torch.float16, device="cuda")
+            ws = H.alloc_workspace(B.OP_GEMV, 1, c.K, c.N, BITS, GROUP)
+            entry.append((c.K, c.N, packed, dev["x"], y, ws))
+            del dev["codes"]
+        sets.append(entry)
+    torch.cuda.synchronize()
+    resident_mb = sum(e[2].numel() for s in sets for e in s) / 1e6
+
+    def step(si):
+        for (K, N, packed, x, y, ws) in sets[si % NSETS]:
+            B.tman_mpgemv(packed, x, y, 1, K, N, BITS, GROUP, ws)
+
+    wbytes_step = sum(weight_bytes(K, N, BITS, GROUP) for _, K, N in MLP)
+    abytes_step = sum(total_bytes(1, K, N, BITS, GROUP) for _, K, N in MLP)
+    launches_per_step = len(MLP)
+
+    # graph of GRAPH_STEPS consecutive steps (launch-bound otherwise: a step is ~10 us of GPU time)
+    for i in range(3):
+        step(i)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(GRAPH_STEPS):
+            step(i)
+    n_replay = max(1, args.steps // GRAPH_STEPS)
+    steps = n_replay * GRAPH_STEPS
+    n_warm = max(1, -(-max(args.warmup, 3) // GRAPH_STEPS))
+    for _ in range(n_warm):
+        graph.replay()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(physical_gpu_index(local_rank)) as clk:
+        ev0.record()
+        for _ in range(n_replay):
+            graph.replay()
+        ev1.record()
+        torch.cuda.synchronize()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    sec_step = ms / 1e3 / steps
+    value = world * wbytes_step / sec_step / 1e9
+    st = [B.tman_read_status(e[5]) for s in sets for e in s]
+    assert all(v == 0 for v in st), f"device status {st}"
+
+    # ---- end to end through the C ABI with host buffers ---------------------------------------
+    xs_host = [torch.from_numpy(c.x.view(np.int16)).view(torch.float16).pin_memory() for c in host0]
+    ys_host = [torch.empty((1, c.N), dtype=torch.float16).pin_memory() for c in host0]
+    h2d = sum(t.numel() * 2 for t in xs_host)
+    d2h = sum(t.numel() * 2 for t in ys_host)
+
+    def e2e_step(si):
+        for j, (K, N, packed, x, y, ws) in enumerate(sets[si % NSETS]):
+            x.copy_(xs_host[j], non_blocking=True)
+            B.tman_mpgemv(packed, x, y, 1, K, N, BITS, GROUP, ws)
+            ys_host[j].copy_(y, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_steps = min(2000, max(50, steps // 10))
+    for i in range(20):
+        e2e_step(i)
+    barrier()
+    ev0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    ev1.record()
+    torch.cuda.synchronize()
+    e2e_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_val = world * wbytes_step / (e2e_ms / 1e3 / e2e_steps) / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": n_warm * GRAPH_STEPS, "ms_per_step": sec_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "replicas": world,
+                   "l2": f"inputs larger than L2: {NSETS} rotating weight sets, {resident_mb:.0f} MB resident",
+                   "launch": f"CUDA graph of {GRAPH_STEPS} steps",
+                   "total_bytes_gbs": world * abytes_step / sec_step / 1e9,
+                   "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS},
+        "clocks": clk.summary(),
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "note": "weights resident; activations copied in and results read back every step"},
+        "gpu_launches": steps * launches_per_step,
+    }
+    avg_launch_s = sec_step / launches_per_step
+    ach = (abytes_step / launches_per_step) / avg_launch_s / 1e9
+    line["roofline"] = {"bound": "hbm", "kernel": "mpgemv_kernel<2,1,8>", "achieved": ach, "peak": peaks["hbm"],
+                        "unit": "GB/s", "frac": ach / peaks["hbm"], "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                        "peak_source": f"of {peaks['src']}", "algorithmic_bytes_per_launch": abytes_step / launches_per_step}
+
+    if rank == 0 and not args.skip_gemm:
+        line["mpgemm"] = bench_gemm(torch, B, H, synth, peaks)
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        line["cpu_baseline"] = cpu_baseline(host0, sets[0])
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists)
+TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def bench_gemm(torch, B, H, synth, peaks):
+    """Prefill mpGEMM, config 4: M=1024, K=4096, N in {4096, 14336}, 4-bit, group 128."""
+    out = {"unit": "TFLOP/s", "cases": []}
+    tot_flops, tot_sec = 0.0, 0.0
+    for spec in synth.config4_specs():
+        c = synth.case_from_spec(spec)
+        dev = H.device_case(c)
+        packed = H.pack_case(c, dev)
+        ncopies = 4
+        xs = [dev["x"].clone() for _ in range(ncopies)]
+        ys = [torch.empty((c.M, c.N), dtype=torch.float16, device="cuda") for _ in range(ncopies)]
+        pks = [packed.clone() for _ in range(ncopies)]
+        ws = H.alloc_workspace(B.OP_GEMM, c.M, c.K, c.N, c.bits, c.group)
+        for i in range(4):
+            B.tman_mpgemm(pks[i % ncopies], xs[i % ncopies], ys[i % ncopies], c.M, c.K, c.N, c.bits, c.group, ws)
+        torch.cuda.synchronize()
+        iters = 40
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            B.tman_mpgemm(pks[i % ncopies], xs[i % ncopies], ys[i % ncopies], c.M, c.K, c.N, c.bits, c.group, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        assert B.tman_read_status(ws) == 0
+        sec = e0.elapsed_time(e1) / 1e3 / iters
+        flops = 2.0 * c.M * c.K * c.N
+        out["cases"].append({"M": c.M, "K": c.K, "N": c.N, "bits": c.bits, "group": c.group,
+                             "us": sec * 1e6, "tflops": flops / sec / 1e12})
+        tot_flops += flops
+        tot_sec += sec
+    tf = tot_flops / tot_sec / 1e12
+    out["value"] = tf
+    out["frac_of_nominal_fp16"] = tf / NOMINAL_FP16_TFLOPS
+    out["roofline"] = {"bound": "tensor", "kernel": "mpgemm_kernel<4>", "achieved": tf, "peak": peaks["tf_burst"],
+                       "unit": "TFLOP/s", "frac": tf / peaks["tf_burst"], "traffic": None,
+                       "peak_source": f"of {peaks['src']} (bf16 burst; fp16 has the same nominal rate)"}
+    return out
+
+
+def cpu_baseline(host0, set0):
+    """The oracle, as it stands, on the host cores: a bounded sample of the same step; also the
+    parity of the timed configuration against it."""
+    from oracle import tman_oracle as orc
+    import torch
+    n_cols = 14336
+    t_probe, _ = time_oracle(host0, 1024, 1, 0)
+    reps = int(max(1, min(20, 10.0 / max(t_probe * 14, 1e-3))))
+    sec, wb = time_oracle(host0, n_cols, reps, 1)
+    outs = oracle_step_sample(host0, n_cols)
+    errs = []
+    for ref, (K, N, packed, x, y, ws) in zip(outs, set0):
+        got = y.detach().cpu().to(torch.float64).numpy()
+        errs.append(float(np.max(np.abs(got - ref)) / np.max(np.abs(ref))))
+    return {"value": wb / sec / 1e9, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{reps} full steps (all columns of the 3 matrices), {sec * 1e3:.1f} ms per step",
+            "parity_max_rel_err": max(errs)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=12000)
+    ap.add_argument("--warmup", type=int, default=600)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--skip-gemm", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
