@@ -95,13 +95,17 @@ tman_status tman_unpack_weights(const void *packed, size_t packed_bytes,
                                 uint8_t *codes, void *scales_f16, uint8_t *zeros,
                                 void *workspace, size_t ws_bytes, tman_stream_t stream);
 
-/* ---- the two matmuls:  y[M][N] (fp16, row-major) = x[M][K] (fp16, row-major) . W ---------- */
+/* ---- the two matmuls:  y[M][N] (fp16, row-major) = x[M][K] (fp16, row-major) . W ----------
+ * packed_bytes is the size of the caller's packed allocation; it must be at least
+ * tman_packed_bytes(K, N, bits, group) (else TMAN_ERR_BUFFER_TOO_SMALL).  With that guarantee the
+ * kernels may start streaming weights before the header check has completed; a header that does
+ * not match the arguments still leaves y untouched and sets the status word. */
 
 /* Decode (paper Sec. 2.2 "Bit-serial table lookup", Fig. 2; Sec. 4.3): activation tables are
  * built in shared memory, packed bit-plane bytes index them, partial sums are
  * shift-accumulated per quantization block, scaled, and summed across blocks in fp32.
  * M in [1, 8]. */
-tman_status tman_mpgemv(const void *packed, const void *x_f16, void *y_f16,
+tman_status tman_mpgemv(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream);
 
@@ -109,7 +113,7 @@ tman_status tman_mpgemv(const void *packed, const void *x_f16, void *y_f16,
  * Fig. 9): packed tiles are staged in shared memory, rebuilt into fp16 tiles through the
  * repack step and the per-(block, column) conversion table, and multiplied on the tensor
  * cores with fp32 accumulation.  M >= 1. */
-tman_status tman_mpgemm(const void *packed, const void *x_f16, void *y_f16,
+tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream);
 

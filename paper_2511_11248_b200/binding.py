@@ -53,8 +53,8 @@ def lib() -> C.CDLL:
         L.tman_read_status.argtypes = [vp, C.POINTER(i), vp]
         L.tman_pack_weights.argtypes = [vp, vp, vp, i, i, i, i, vp, sz, vp]
         L.tman_unpack_weights.argtypes = [vp, sz, i, i, i, i, vp, vp, vp, vp, sz, vp]
-        L.tman_mpgemv.argtypes = [vp, vp, vp, i, i, i, i, i, vp, sz, vp]
-        L.tman_mpgemm.argtypes = [vp, vp, vp, i, i, i, i, i, vp, sz, vp]
+        L.tman_mpgemv.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, sz, vp]
+        L.tman_mpgemm.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, sz, vp]
         L.tman_debug_indices.argtypes = [vp, i, i, i, i, vp, vp, sz, vp]
         L.tman_debug_luts.argtypes = [vp, i, i, vp, vp]
         for name in EXPORTS[2:]:
@@ -124,13 +124,13 @@ def tman_unpack_weights(packed, K, N, bits, group, codes, scales, zeros, workspa
 
 
 def tman_mpgemv(packed, x, y, M, K, N, bits, group, workspace, stream=None) -> None:
-    _check(lib().tman_mpgemv(_ptr(packed), _ptr(x), _ptr(y), M, K, N, bits, group, _ptr(workspace),
+    _check(lib().tman_mpgemv(_ptr(packed), packed.numel() * packed.element_size(), _ptr(x), _ptr(y), M, K, N, bits, group, _ptr(workspace),
                              workspace.numel() * workspace.element_size(), _stream(stream)),
            "tman_mpgemv")
 
 
 def tman_mpgemm(packed, x, y, M, K, N, bits, group, workspace, stream=None) -> None:
-    _check(lib().tman_mpgemm(_ptr(packed), _ptr(x), _ptr(y), M, K, N, bits, group, _ptr(workspace),
+    _check(lib().tman_mpgemm(_ptr(packed), packed.numel() * packed.element_size(), _ptr(x), _ptr(y), M, K, N, bits, group, _ptr(workspace),
                              workspace.numel() * workspace.element_size(), _stream(stream)),
            "tman_mpgemm")
 

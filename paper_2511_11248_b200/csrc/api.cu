@@ -97,23 +97,24 @@ tman_status tman_unpack_weights(const void *packed, size_t packed_bytes,
                          static_cast<uint32_t *>(workspace), reinterpret_cast<cudaStream_t>(stream));
 }
 
-static tman_status check_matmul(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
-                                int group, void *ws)
+static tman_status check_matmul(const void *packed, size_t packed_bytes, const void *x, void *y, int M, int K,
+                                int N, int bits, int group, void *ws)
 {
     if (!packed || !x || !y || !ws) return TMAN_ERR_NULL;
     tman_status st = check_format(K, N, bits, group);
     if (st != TMAN_OK) return st;
+    if (packed_bytes < make_layout(K, N, bits, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
     if (bits < 2) return TMAN_ERR_UNSUPPORTED;
     if (M < 1) return TMAN_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(packed) & 255) return TMAN_ERR_SHAPE;
     return TMAN_OK;
 }
 
-tman_status tman_mpgemv(const void *packed, const void *x_f16, void *y_f16,
+tman_status tman_mpgemv(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream)
 {
-    tman_status st = check_matmul(packed, x_f16, y_f16, M, K, N, bits, group, workspace);
+    tman_status st = check_matmul(packed, packed_bytes, x_f16, y_f16, M, K, N, bits, group, workspace);
     if (st != TMAN_OK) return st;
     if (M > 8) return TMAN_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(x_f16) & 15) return TMAN_ERR_SHAPE;
@@ -122,11 +123,11 @@ tman_status tman_mpgemv(const void *packed, const void *x_f16, void *y_f16,
                          reinterpret_cast<cudaStream_t>(stream));
 }
 
-tman_status tman_mpgemm(const void *packed, const void *x_f16, void *y_f16,
+tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream)
 {
-    tman_status st = check_matmul(packed, x_f16, y_f16, M, K, N, bits, group, workspace);
+    tman_status st = check_matmul(packed, packed_bytes, x_f16, y_f16, M, K, N, bits, group, workspace);
     if (st != TMAN_OK) return st;
     if (ws_bytes < mpgemm_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
     return launch_mpgemm(packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,

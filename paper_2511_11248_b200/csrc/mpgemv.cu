@@ -21,6 +21,22 @@
 
 namespace tman {
 
+// Optional phase time stamps for experiments (compiled out of the library build).
+#ifdef TMAN_PHASE_TIMERS
+__device__ unsigned long long *tman_stamp_buf;
+#define TMAN_STAMP(i)                                                              \
+    do {                                                                           \
+        if (threadIdx.x == 0) {                                                    \
+            unsigned long long t_;                                                 \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                 \
+            tman_stamp_buf[blockIdx.x * 16 + (i)] = t_;                            \
+            tman_stamp_buf[blockIdx.x * 16 + 8 + (i)] = (unsigned long long)clock64(); \
+        }                                                                          \
+    } while (0)
+#else
+#define TMAN_STAMP(i) do {} while (0)
+#endif
+
 constexpr int kGemvThreads = 512;
 constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kGemvTableBytes = 128 * 1024;   // 4 groups x 256 entries x 32 slots x 4 B
@@ -93,11 +109,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     constexpr int V = 4 * S * MT;         // values a lane produces per warp-unit
     constexpr int NKEEP = (V >= W) ? V / W : 1;
 
-    if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {
-        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
-        return;
-    }
-
+    TMAN_STAMP(0);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kappa = blockIdx.x / p.P, j = blockIdx.x % p.P;
     const int words_total = p.K / 32;
@@ -108,6 +120,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     const int nstrips = p.N / 4;
     const int nblk = p.K / p.group;
     const int B = active ? ((word0 + v) * 32) / p.group : 0;
+
+    // Let the next kernel in the stream start its own weight streaming while this one drains
+    // (programmatic dependent launch); the header words are requested now and checked later.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    uint32_t hdr[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) hdr[q] = __ldg(reinterpret_cast<const uint32_t *>(p.packed) + q);
 
     uint4    wreg[S][BITS];
     uint2    sreg[S];
@@ -134,31 +153,43 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         }
     };
 
-    // issue the first unit's weight loads before building the tables: their latency overlaps
+    // Issue the first unit's weight loads before anything else: the packed buffer is constant
+    // input and packed_bytes was checked on the host, so these reads are in bounds whatever the
+    // header says.  Their latency overlaps the table build.
     int wu = j + p.P * warp;
     if (wu < p.units) load_unit(wu);
+    TMAN_STAMP(1);
+
+    // Everything below may depend on the previous kernel in the stream (activations, workspace).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // The activations of this thread's table slot (one plane word = 32 activations of one row).
+    const int vb = lane / MT, mb = lane % MT;
+    const bool live = (vb < nwords) && (mb < p.M);
+    uint4 xraw[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) xraw[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (live) {
+        const uint4 *px = reinterpret_cast<const uint4 *>(p.x + (size_t)mb * p.K + (size_t)(word0 + vb) * 32);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) xraw[c] = __ldg(px + c);
+    }
+    TMAN_STAMP(2);
 
     // ---- phase A: activation tables (paper Sec. 2.2; one table per 8 activations, 256 entries,
     // entry = 16-entry table of the low four + sum of the selected high four) -----------------
     {
-        const int vb = lane / MT, mb = lane % MT;
-        const bool live = (vb < nwords) && (mb < p.M);
-#pragma unroll 1
-        for (int task = warp; task < 64; task += kGemvWarps) {
-            const int c = task >> 4, ph = task & 15;
+        // warp w fills the entries whose high index nibble is w, for all four groups of the word
+        const int ph = warp;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
             float xv[8];
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&xraw[c]);
 #pragma unroll
-            for (int q = 0; q < 8; ++q) xv[q] = 0.f;
-            if (live) {
-                const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(
-                    p.x + (size_t)mb * p.K + (size_t)(word0 + vb) * 32 + 8 * c));
-                const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    float2 f = __half22float2(h2[q]);
-                    xv[2 * q] = f.x;
-                    xv[2 * q + 1] = f.y;
-                }
+            for (int q = 0; q < 4; ++q) {
+                const float2 f = __half22float2(h2[q]);
+                xv[2 * q] = f.x;
+                xv[2 * q + 1] = f.y;
             }
             float lo[16];
             lut16(xv[0], xv[1], xv[2], xv[3], lo);
@@ -174,6 +205,18 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         }
     }
     __syncthreads();
+    TMAN_STAMP(3);
+
+    // header check (uniform over the grid): a mismatch leaves every output untouched
+    {
+        const bool hdr_ok = (hdr[0] == 0x4E414D54u) && (hdr[1] == 0x30303242u) && (hdr[2] == kVersion) &&
+                            (hdr[3] == (uint32_t)p.K) && (hdr[4] == (uint32_t)p.N) &&
+                            (hdr[5] == (uint32_t)p.bits) && (hdr[6] == (uint32_t)p.group) && (hdr[7] == 4u);
+        if (!hdr_ok) {
+            if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
+            return;
+        }
+    }
 
     // the lane's activation sum over its 32 activations (all-ones entries), for the zero-point term
     const uint32_t sub_off = (uint32_t)(v * MT * 4);
@@ -228,11 +271,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             }
         }
 
+        TMAN_STAMP(4);
         // ---- reduce the K-slice's lanes (warp shuffles) -----------------------------------------
         int base = 0;
         LaneReduce<V, W / 2>::run(vals, v, base);
         const bool writer = (V >= W) ? true : ((v & (W / V - 1)) == 0);
         const int col0 = (wu * MT + sub) * S * 4;      // first column of this sub-warp's strips
+        TMAN_STAMP(5);
 
         if (p.nkappa == 1) {
             if (writer) {
@@ -256,6 +301,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             uint32_t old = 0;
             if (lane == 0) old = atomicAdd(p.counters + wu, 1u);
             old = __shfl_sync(0xffffffffu, old, 0);
+            TMAN_STAMP(6);
             if (old == (uint32_t)(p.nkappa - 1)) {
                 __threadfence();
                 constexpr int C = 4 * S * MT;           // columns of the warp-unit
@@ -273,6 +319,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             }
         }
     }
+    TMAN_STAMP(7);
 }
 
 template <int BITS, int MT>
@@ -293,8 +340,18 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     auto kern = mpgemv_kernel<BITS, MT, S>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvTableBytes) != cudaSuccess)
         return TMAN_ERR_CUDA;
-    kern<<<p.nkappa * p.P, kGemvThreads, kGemvTableBytes, s>>>(p);
-    return launch_status();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.nkappa * p.P));
+    cfg.blockDim = dim3(kGemvThreads);
+    cfg.dynamicSmemBytes = kGemvTableBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) return TMAN_ERR_CUDA;
+    return TMAN_OK;
 }
 
 template <int BITS>

@@ -79,16 +79,18 @@ def test_null_and_range_errors_before_any_launch(lib):
     assert lib.tman_workspace_bytes(0, 0, 128, 8, 4, 64, C.byref(out)) == 2
     # null data pointers: rejected on the host
     assert lib.tman_pack_weights(None, None, None, 128, 8, 4, 64, None, 0, None) == 1
-    assert lib.tman_mpgemv(None, None, None, 1, 128, 8, 4, 64, None, 0, None) == 1
-    assert lib.tman_mpgemm(None, None, None, 1, 128, 8, 4, 64, None, 0, None) == 1
+    assert lib.tman_mpgemv(None, 0, None, None, 1, 128, 8, 4, 64, None, 0, None) == 1
+    assert lib.tman_mpgemm(None, 0, None, None, 1, 128, 8, 4, 64, None, 0, None) == 1
     assert lib.tman_debug_luts(None, 1, 128, None, None) == 1
     # fake non-null pointers (never dereferenced: the size checks fail first)
     fake = C.c_void_p(4096 * 256)
     assert lib.tman_pack_weights(fake, fake, fake, 128, 8, 4, 64, fake, 16, None) == 4
-    assert lib.tman_mpgemv(fake, fake, fake, 9, 128, 8, 4, 64, fake, 1 << 30, None) == 2
-    assert lib.tman_mpgemv(fake, fake, fake, 1, 128, 8, 1, 64, fake, 1 << 30, None) == 3
-    assert lib.tman_mpgemv(fake, fake, fake, 1, 128, 8, 4, 64, fake, 8, None) == 4
-    assert lib.tman_mpgemm(fake, fake, fake, 0, 128, 8, 4, 64, fake, 1 << 30, None) == 2
+    assert lib.tman_mpgemv(fake, 1 << 30, fake, fake, 9, 128, 8, 4, 64, fake, 1 << 30, None) == 2
+    assert lib.tman_mpgemv(fake, 1 << 30, fake, fake, 1, 128, 8, 1, 64, fake, 1 << 30, None) == 3
+    assert lib.tman_mpgemv(fake, 1 << 30, fake, fake, 1, 128, 8, 4, 64, fake, 8, None) == 4
+    assert lib.tman_mpgemv(fake, 300, fake, fake, 1, 128, 8, 4, 64, fake, 1 << 30, None) == 4
+    assert lib.tman_mpgemm(fake, 300, fake, fake, 1, 128, 8, 4, 64, fake, 1 << 30, None) == 4
+    assert lib.tman_mpgemm(fake, 1 << 30, fake, fake, 0, 128, 8, 4, 64, fake, 1 << 30, None) == 2
     assert lib.tman_unpack_weights(fake, 16, 128, 8, 4, 64, fake, fake, fake, fake, 256, None) == 4
     assert lib.tman_workspace_init(fake, 8, None) == 4
 
