@@ -117,6 +117,31 @@ tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream);
 
+/* Decode without a caller-supplied workspace.  (No counterpart in the paper: this call exists for
+ * the way the library is embedded, not for the method.)
+ *
+ * For callers that may not allocate device memory when they need a matmul -- a runtime that fixed
+ * its arena at start-up, code running inside another framework's callback, a region where the
+ * allocator is locked -- and so cannot produce the workspace tman_mpgemv asks for.  The scratch
+ * is a fixed 4 MiB array inside the library image; every GPU that loads the library holds it
+ * until the process exits, and this call allocates and frees nothing.
+ *
+ *   - Same result as tman_mpgemv for the same arguments (same kernels, same summation order).
+ *   - A shape whose scratch, tman_workspace_bytes(0, M, K, N, bits, group), exceeds 4 MiB is
+ *     refused with TMAN_ERR_BUFFER_TOO_SMALL before anything is enqueued.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents: each
+ *     call first clears the part that must start at zero.  Two calls that overlap on the GPU
+ *     (different streams without an ordering between them) race on it and give wrong results;
+ *     calls on one stream, or ordered by events, are fine.
+ *   - status_dev: device pointer to 4 bytes owned by the caller, or NULL.  When given, the
+ *     device-side status word (0, TMAN_ERR_BAD_PACKED, ...) is copied there on `stream` after the
+ *     kernels. */
+tman_status tman_mpgemv_static(const void *packed, size_t packed_bytes, const void *x_f16,
+                               void *y_f16, int M, int K, int N, int bits, int group,
+                               unsigned int *status_dev, tman_stream_t stream);
+
 /* ---- test-only extractors of the integer / table intermediates -------------------------- */
 
 /* idx uint8 [bits][K/4][N]: the 4-bit table index of every (plane, 4 activations, column)

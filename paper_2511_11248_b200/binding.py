@@ -22,7 +22,7 @@ OP_GEMV, OP_GEMM, OP_AUX = 0, 1, 2
 EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
-    "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts",
+    "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_mpgemv_static",
 ]
 
 _lib = None
@@ -55,6 +55,7 @@ def lib() -> C.CDLL:
         L.tman_unpack_weights.argtypes = [vp, sz, i, i, i, i, vp, vp, vp, vp, sz, vp]
         L.tman_mpgemv.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, sz, vp]
         L.tman_mpgemm.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, sz, vp]
+        L.tman_mpgemv_static.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, vp]
         L.tman_debug_indices.argtypes = [vp, i, i, i, i, vp, vp, sz, vp]
         L.tman_debug_luts.argtypes = [vp, i, i, vp, vp]
         for name in EXPORTS[2:]:
@@ -127,6 +128,14 @@ def tman_mpgemv(packed, x, y, M, K, N, bits, group, workspace, stream=None) -> N
     _check(lib().tman_mpgemv(_ptr(packed), packed.numel() * packed.element_size(), _ptr(x), _ptr(y), M, K, N, bits, group, _ptr(workspace),
                              workspace.numel() * workspace.element_size(), _stream(stream)),
            "tman_mpgemv")
+
+
+def tman_mpgemv_static(packed, x, y, M, K, N, bits, group, status=None, stream=None) -> None:
+    """Decode matmul on the library's built-in scratch array: for callers that cannot allocate a
+    workspace.  `status`, if given, is a 4-byte device tensor that receives the device-side status."""
+    _check(lib().tman_mpgemv_static(_ptr(packed), packed.numel() * packed.element_size(), _ptr(x), _ptr(y),
+                                    M, K, N, bits, group, _ptr(status), _stream(stream)),
+           "tman_mpgemv_static")
 
 
 def tman_mpgemm(packed, x, y, M, K, N, bits, group, workspace, stream=None) -> None:

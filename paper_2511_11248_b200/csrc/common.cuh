@@ -112,6 +112,7 @@ tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int
                                  uint32_t *status, cudaStream_t s);
 tman_status launch_debug_luts(const void *x, int M, int K, float *lut, cudaStream_t s);
 size_t      mpgemv_workspace_bytes(int M, int K, int N);
+size_t      mpgemv_workspace_zero_prefix(int N);
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s);
 size_t      mpgemm_workspace_bytes(int M, int K, int N);

@@ -371,6 +371,9 @@ size_t mpgemv_workspace_bytes(int M, int K, int N)
     return kWsStatusBytes + ws_counter_bytes(N) + nkappa * 4 * (size_t)N * sizeof(float);
 }
 
+// bytes at the start of a workspace that must be zero before a call (status word and counters)
+size_t mpgemv_workspace_zero_prefix(int N) { return kWsStatusBytes + ws_counter_bytes(N); }
+
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s)
 {
