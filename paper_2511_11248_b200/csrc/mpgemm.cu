@@ -23,14 +23,15 @@
 namespace tman {
 namespace {
 
+// A CTA multiplies MH row blocks of 128 tokens by one dequantized 128-column weight tile: every
+// weight is rebuilt once per 128*MH tokens (MH = 2 halves the dequantization work per flop).
 constexpr int BM = 128, BN = 128, BK = 64;
 constexpr int NSTAGE = 4;
-constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int A_HALF_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_DEQ_WARPS = 8;
 constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS);
-constexpr int TMEM_COLS = 128;
-constexpr int SMEM_BYTES = NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int smem_bytes(int mh) { return NSTAGE * (mh * A_HALF_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/; }
 
 struct GemmParams {
     const uint8_t  *packed;
@@ -243,10 +244,12 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
         }
 }
 
-template <int BITS>
+template <int BITS, int MH>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
 {
+    constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
+    constexpr int TMEM_COLS = MH * BN;                 // one fp32 accumulator of BN columns per row block
     extern __shared__ uint8_t smem_raw[];
     if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
@@ -293,7 +296,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
                 const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
                 mbar_expect_tx(full0 + 8 * s, A_STAGE_BYTES);
-                tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, tile_m * BM, full0 + 8 * s);
+                tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, tile_m * (BM * MH), full0 + 8 * s);
             }
         }
     } else if (warp == 1) {
@@ -305,11 +308,15 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
                 const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
                 if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
                 tcgen05_fence_after();
-                const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES));
                 const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
 #pragma unroll
                 for (int j = 0; j < BK / 16; ++j)
-                    tcgen05_mma_f16(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc, (kb > 0 || j > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int h = 0; h < MH; ++h) {
+                        const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES + h * A_HALF_BYTES));
+                        tcgen05_mma_f16(tmem_base + (uint32_t)(h * BN), adesc + 2 * j, bdesc + 2 * j, idesc,
+                                        (kb > 0 || j > 0) ? 1u : 0u);
+                    }
                 tcgen05_commit(empty0 + 8 * s);
             }
             if (ok) tcgen05_commit(accum_bar);
@@ -378,12 +385,13 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
             tcgen05_fence_after();
             const int quarter = warp & 3;                 // tensor-memory lanes this warp may read
             const int col_half = wd >> 2;                 // columns [0,64) or [64,128)
-            const int m = tile_m * BM + quarter * 32 + lane;
 #pragma unroll 1
-            for (int cc = 0; cc < 2; ++cc) {
+            for (int hc = 0; hc < 2 * MH; ++hc) {
+                const int h = hc >> 1, cc = hc & 1;
+                const int m = tile_m * (BM * MH) + h * BM + quarter * 32 + lane;
                 const int col = col_half * 64 + cc * 32;
                 uint32_t r[32];
-                tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, r);
+                tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * BN + col), r);
                 tcgen05_wait_ld();
                 if (m < p.M) {
                     __half *dst = p.y + (size_t)m * p.N + (size_t)tile_n * BN + col;
@@ -429,14 +437,20 @@ EncodeTiledFn encode_fn()
     return reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-template <int BITS>
-tman_status launch_bits(const CUtensorMap &tmap, const GemmParams &p, cudaStream_t s)
+template <int BITS, int MH>
+tman_status launch_tile(const CUtensorMap &tmap, const GemmParams &p, cudaStream_t s)
 {
-    auto kern = mpgemm_kernel<BITS>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+    auto kern = mpgemm_kernel<BITS, MH>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(MH)) != cudaSuccess)
         return TMAN_ERR_CUDA;
-    kern<<<p.tiles_m * p.tiles_n, GEMM_THREADS, SMEM_BYTES, s>>>(tmap, p);
+    kern<<<p.tiles_m * p.tiles_n, GEMM_THREADS, smem_bytes(MH), s>>>(tmap, p);
     return launch_status();
+}
+
+template <int BITS>
+tman_status launch_bits(const CUtensorMap &tmap, const GemmParams &p, int mh, cudaStream_t s)
+{
+    return mh == 2 ? launch_tile<BITS, 2>(tmap, p, s) : launch_tile<BITS, 1>(tmap, p, s);
 }
 
 }  // namespace
@@ -452,7 +466,8 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     CUtensorMap tmap;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    const int mh = (M > BM) ? 2 : 1;                   // row blocks per CTA
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)(BM * mh)};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(x), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -469,11 +484,11 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.y = static_cast<__half *>(y);
     p.status = static_cast<uint32_t *>(ws);
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
-    p.tiles_m = (M + BM - 1) / BM;
+    p.tiles_m = (M + BM * mh - 1) / (BM * mh);
     p.tiles_n = (N + BN - 1) / BN;
-    if (bits == 2) return launch_bits<2>(tmap, p, s);
-    if (bits == 3) return launch_bits<3>(tmap, p, s);
-    return launch_bits<4>(tmap, p, s);
+    if (bits == 2) return launch_bits<2>(tmap, p, mh, s);
+    if (bits == 3) return launch_bits<3>(tmap, p, mh, s);
+    return launch_bits<4>(tmap, p, mh, s);
 }
 
 }  // namespace tman
