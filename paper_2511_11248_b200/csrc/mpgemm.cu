@@ -4,8 +4,9 @@
 //
 // One CTA computes a 128 x 128 tile of y.  Three kinds of agents run concurrently on a ring of
 // shared-memory stages guarded by mbarriers (the paper's DMA / vector-core / matrix-core stages):
-//   * warp 0, one lane : TMA loads of the fp16 activation tile (128 x 64, 128-byte swizzle);
-//   * warps 2..9       : read the packed bit-plane words of their column, rebuild the codes
+//   * warp 0, one lane : TMA loads of the fp16 activation tile (128-byte swizzle) and of the packed
+//                        bit-plane words of the weight tile (one box per plane);
+//   * warps 2..9       : read the staged plane words of their column, rebuild the codes
 //                        (level 1: bit-serial -> bit-parallel), look every code up in the
 //                        per-(block, column) conversion table kept in registers and addressed
 //                        with byte-permute instructions (level 2: scale and zero-point baked in),
@@ -31,7 +32,11 @@ constexpr int A_HALF_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_DEQ_WARPS = 8;
 constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS);
-constexpr int smem_bytes(int mh) { return NSTAGE * (mh * A_HALF_BYTES + B_STAGE_BYTES) + 1024 /*align*/ + 256 /*barriers*/; }
+constexpr int P_PLANE_BYTES = (BN / 4) * (BK / 32) * 16;       // one plane of a packed tile: 32 strips x 2 words x 16 B
+constexpr int smem_bytes(int mh, int bits)
+{
+    return NSTAGE * (mh * A_HALF_BYTES + B_STAGE_BYTES + bits * P_PLANE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+}
 
 struct GemmParams {
     const uint8_t  *packed;
@@ -101,6 +106,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tma
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tmap, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tcgen05_alloc(uint32_t dst_smem, uint32_t ncols)
 {
@@ -173,14 +184,18 @@ struct ConvTable {
     static constexpr int NQ = (BITS == 4) ? 4 : ((BITS == 3) ? 2 : 1);
     uint32_t lo[NQ], hi[NQ];
 
+    // entry c = fp16(s * (c - z)): c - z is a small integer (exact in fp16), so one half-precision
+    // multiply rounds once, like the fp32 product rounded to fp16 would
     __device__ __forceinline__ void build(__half s, uint32_t z)
     {
-        const float sf = __half2float(s);
-        const float nsz = -sf * (float)z;
+        const __half2 s2 = __half2half2(s);
+        const __half2 z2 = __half2half2(__ushort2half_rn((unsigned short)z));
 #pragma unroll
         for (int q = 0; q < NQ; ++q) {
-            const __half2 e01 = __floats2half2_rn(fmaf(sf, (float)(4 * q + 0), nsz), fmaf(sf, (float)(4 * q + 1), nsz));
-            const __half2 e23 = __floats2half2_rn(fmaf(sf, (float)(4 * q + 2), nsz), fmaf(sf, (float)(4 * q + 3), nsz));
+            const __half2 c01 = __floats2half2_rn((float)(4 * q + 0), (float)(4 * q + 1));
+            const __half2 c23 = __floats2half2_rn((float)(4 * q + 2), (float)(4 * q + 3));
+            const __half2 e01 = __hmul2(s2, __hsub2(c01, z2));
+            const __half2 e23 = __hmul2(s2, __hsub2(c23, z2));
             const uint32_t h01 = *reinterpret_cast<const uint32_t *>(&e01);
             const uint32_t h23 = *reinterpret_cast<const uint32_t *>(&e23);
             lo[q] = __byte_perm(h01, h23, 0x6420);
@@ -213,14 +228,27 @@ struct ConvTable {
 template <int BITS>
 __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const ConvTable<BITS> &T, uint32_t (&out)[16])
 {
-    // level 1 (bit repacking): X[ph] nibble j = code of weight 4j + ph
+    // level 1 (bit repacking): X[ph] nibble j = code of weight 4j + ph.  A 4 x 4 bit-block
+    // transpose of the plane words: first planes 0/1 and 2/3 are interleaved bit by bit, then the
+    // two results two bits by two bits (each step is one shift and one bit-select).
+    auto bsel = [](uint32_t m, uint32_t a, uint32_t b) { return (a & m) | (b & ~m); };
     uint32_t X[4];
-#pragma unroll
-    for (int ph = 0; ph < 4; ++ph) {
-        uint32_t x = 0;
-#pragma unroll
-        for (int i = 0; i < BITS; ++i) x |= ((w[i] >> ph) & 0x11111111u) << i;
-        X[ph] = x;
+    {
+        const uint32_t w0 = w[0], w1 = w[1];
+        const uint32_t a0 = bsel(0x55555555u, w0, w1 << 1), a1 = bsel(0x55555555u, w0 >> 1, w1);
+        if constexpr (BITS > 2) {
+            const uint32_t w2 = w[2], w3 = (BITS > 3) ? w[BITS - 1] : 0u;
+            const uint32_t b0 = bsel(0x55555555u, w2, w3 << 1), b1 = bsel(0x55555555u, w2 >> 1, w3);
+            X[0] = bsel(0x33333333u, a0, b0 << 2);
+            X[2] = bsel(0x33333333u, a0 >> 2, b0);
+            X[1] = bsel(0x33333333u, a1, b1 << 2);
+            X[3] = bsel(0x33333333u, a1 >> 2, b1);
+        } else {
+            X[0] = a0 & 0x33333333u;
+            X[2] = (a0 >> 2) & 0x33333333u;
+            X[1] = a1 & 0x33333333u;
+            X[3] = (a1 >> 2) & 0x33333333u;
+        }
     }
     // level 2 (conversion table) and re-pairing into adjacent k
     uint32_t A[4][2], Bv[4][2];
@@ -246,10 +274,11 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
 
 template <int BITS, int MH>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
+mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const GemmParams p)
 {
     constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
     constexpr int TMEM_COLS = MH * BN;                 // one fp32 accumulator of BN columns per row block
+    constexpr int P_STAGE_BYTES = BITS * P_PLANE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
@@ -258,20 +287,24 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *a_tiles = smem;
     uint8_t *b_tiles = smem + NSTAGE * A_STAGE_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES));
-    // bars[0..NSTAGE) full, [NSTAGE..2NSTAGE) empty, [2NSTAGE] accumulator ready
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * NSTAGE + 1);
+    uint8_t *p_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + P_STAGE_BYTES));
+    // bars[0..NSTAGE) loaded (TMA), [NSTAGE..2NSTAGE) full (dequantized), [2NSTAGE..3NSTAGE) empty,
+    // [3NSTAGE] accumulator ready
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * NSTAGE + 1);
     uint32_t *fail_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile_m = blockIdx.x % p.tiles_m, tile_n = blockIdx.x / p.tiles_m;
     const int num_kb = p.K / BK;
 
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + NSTAGE), accum_bar = smem_u32(bars + 2 * NSTAGE);
+    const uint32_t loaded0 = smem_u32(bars), full0 = smem_u32(bars + NSTAGE), empty0 = smem_u32(bars + 2 * NSTAGE),
+                   accum_bar = smem_u32(bars + 3 * NSTAGE);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NSTAGE; ++s) {
-            mbar_init(full0 + 8 * s, 1 + NUM_DEQ_WARPS);
+            mbar_init(loaded0 + 8 * s, 1);
+            mbar_init(full0 + 8 * s, NUM_DEQ_WARPS);
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum_bar, 1);
@@ -295,8 +328,12 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
                 const int s = kb % NSTAGE;
                 const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
-                mbar_expect_tx(full0 + 8 * s, A_STAGE_BYTES);
-                tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, tile_m * (BM * MH), full0 + 8 * s);
+                mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + P_STAGE_BYTES);
+                tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, tile_m * (BM * MH), loaded0 + 8 * s);
+#pragma unroll
+                for (int i = 0; i < BITS; ++i)
+                    tma_load_3d(smem_u32(p_tiles + s * P_STAGE_BYTES + i * P_PLANE_BYTES), &tmap_w, kb * (BK / 8), i,
+                                tile_n * (BN / 4), loaded0 + 8 * s);
             }
         }
     } else if (warp == 1) {
@@ -323,50 +360,55 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p)
         }
     } else {
         // ---- stage 2: two-level lookup dequantization ----------------------------------------
+        // A warp owns 16 columns and both plane words of a k-block: lane = (strip of the warp, word,
+        // column of the strip).  With this split the 32 lanes read 32 different banks of the staged
+        // plane words and write eight different 16-byte bank groups per quarter-warp.
         const int wd = warp - 2;
-        const int n_local = (wd & 3) * 32 + lane;
-        const int v = wd >> 2;                         // which of the two plane words of a k-block
+        const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
+        const int n_local = wd * 16 + sl * 4 + c;
         const int n = tile_n * BN + n_local;
         const bool valid = n < p.N;
-        const int nb = n >> 2, c = n & 3;
-        const int words_total = p.K / 32;
+        const int nb = n >> 2;
         const int nblk = p.K / p.group;
-        const uint32_t *wp = p.planes + ((size_t)nb * BITS * words_total) * 4 + c;
+        const int gshift = (p.group == 32) ? 5 : (p.group == 64) ? 6 : 7;
+        const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
         const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
         const uint32_t xr = (uint32_t)(n_local & 7);
+        const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
+        const uint16_t *pz = p.zeros + (size_t)nb * nblk;
 
+        // scale and zero-point of the next quantization block are fetched one block ahead
+        auto fetch_sz = [&](int B, __half &sv, uint32_t &zz) {
+            sv = __float2half(0.f);
+            zz = 0u;
+            if (valid && B < nblk) {
+                sv = __ldg(ps + (size_t)B * 4);
+                zz = ((uint32_t)__ldg(pz + B) >> (4 * c)) & 0xFu;
+            }
+        };
         ConvTable<BITS> T;
         int cur_B = -1;
-        uint32_t wnext[BITS];
-#pragma unroll
-        for (int i = 0; i < BITS; ++i)
-            wnext[i] = valid ? __ldg(wp + ((size_t)i * words_total + v) * 4) : 0u;
+        const int B_step = (p.group == 32) ? 2 : 1;        // this lane's next block
+        __half sv_next;
+        uint32_t zz_next;
+        fetch_sz((v * 32) >> gshift, sv_next, zz_next);
 
         for (int kb = 0; kb < num_kb; ++kb) {
             const int s = kb % NSTAGE;
             const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
-            uint32_t w[BITS];
-#pragma unroll
-            for (int i = 0; i < BITS; ++i) w[i] = wnext[i];
-            if (kb + 1 < num_kb) {
-#pragma unroll
-                for (int i = 0; i < BITS; ++i)
-                    wnext[i] = valid ? __ldg(wp + ((size_t)i * words_total + 2 * (kb + 1) + v) * 4) : 0u;
-            }
-            const int Bk = ((2 * kb + v) * 32) / p.group;
+            const int Bk = ((2 * kb + v) * 32) >> gshift;
             if (Bk != cur_B) {
                 cur_B = Bk;
-                __half sv = __float2half(0.f);
-                uint32_t zz = 0;
-                if (valid) {
-                    sv = __ldg(p.scales + ((size_t)nb * nblk + Bk) * 4 + c);
-                    zz = ((uint32_t)__ldg(p.zeros + (size_t)nb * nblk + Bk) >> (4 * c)) & 0xFu;
-                }
-                T.build(sv, zz);
+                T.build(sv_next, zz_next);
+                fetch_sz(Bk + B_step, sv_next, zz_next);
             }
+            if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
+            uint32_t w[BITS];
+            const uint8_t *pp = p_tiles + s * P_STAGE_BYTES + p_off;
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) w[i] = *reinterpret_cast<const uint32_t *>(pp + i * P_PLANE_BYTES);
             uint32_t out[16];
             dequant_word<BITS>(w, T, out);
-            if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
             uint8_t *row = b_tiles + s * B_STAGE_BYTES + row_off;
 #pragma unroll
             for (int cj = 0; cj < 4; ++cj) {
@@ -438,19 +480,19 @@ EncodeTiledFn encode_fn()
 }
 
 template <int BITS, int MH>
-tman_status launch_tile(const CUtensorMap &tmap, const GemmParams &p, cudaStream_t s)
+tman_status launch_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, cudaStream_t s)
 {
     auto kern = mpgemm_kernel<BITS, MH>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(MH)) != cudaSuccess)
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(MH, BITS)) != cudaSuccess)
         return TMAN_ERR_CUDA;
-    kern<<<p.tiles_m * p.tiles_n, GEMM_THREADS, smem_bytes(MH), s>>>(tmap, p);
+    kern<<<p.tiles_m * p.tiles_n, GEMM_THREADS, smem_bytes(MH, BITS), s>>>(tmap_x, tmap_w, p);
     return launch_status();
 }
 
 template <int BITS>
-tman_status launch_bits(const CUtensorMap &tmap, const GemmParams &p, int mh, cudaStream_t s)
+tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, int mh, cudaStream_t s)
 {
-    return mh == 2 ? launch_tile<BITS, 2>(tmap, p, s) : launch_tile<BITS, 1>(tmap, p, s);
+    return mh == 2 ? launch_tile<BITS, 2>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1>(tmap_x, tmap_w, p, s);
 }
 
 }  // namespace
@@ -476,6 +518,20 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
 
     Layout L = make_layout(K, N, bits, group);
     const uint8_t *pk = static_cast<const uint8_t *>(packed);
+    // the bit-plane words as a 3-D array of 32-bit elements: (word and column inside a strip's plane
+    // row, plane, strip); one box = the two words of a k-block for 32 strips of one plane
+    CUtensorMap tmap_w;
+    {
+        const cuuint64_t wt = (cuuint64_t)(K / 32);
+        const cuuint64_t wdims[3] = {wt * 4, (cuuint64_t)bits, (cuuint64_t)(N / 4)};
+        const cuuint64_t wstrides[2] = {wt * 16, wt * 16 * (cuuint64_t)bits};
+        const cuuint32_t wbox[3] = {(cuuint32_t)(BK / 8), 1, (cuuint32_t)(BN / 4)};
+        const cuuint32_t westr[3] = {1, 1, 1};
+        if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t *>(pk + L.planes_off), wdims, wstrides,
+                wbox, westr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TMAN_ERR_CUDA;
+    }
     GemmParams p;
     p.packed = pk;
     p.planes = reinterpret_cast<const uint32_t *>(pk + L.planes_off);
@@ -486,9 +542,9 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
     p.tiles_m = (M + BM * mh - 1) / (BM * mh);
     p.tiles_n = (N + BN - 1) / BN;
-    if (bits == 2) return launch_bits<2>(tmap, p, mh, s);
-    if (bits == 3) return launch_bits<3>(tmap, p, mh, s);
-    return launch_bits<4>(tmap, p, mh, s);
+    if (bits == 2) return launch_bits<2>(tmap, tmap_w, p, mh, s);
+    if (bits == 3) return launch_bits<3>(tmap, tmap_w, p, mh, s);
+    return launch_bits<4>(tmap, tmap_w, p, mh, s);
 }
 
 }  // namespace tman
