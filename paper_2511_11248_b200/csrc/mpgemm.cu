@@ -374,6 +374,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
         const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
         const uint32_t xr = (uint32_t)(n_local & 7);
+        const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
         const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
         const uint16_t *pz = p.zeros + (size_t)nb * nblk;
 
@@ -404,17 +405,18 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             }
             if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
             uint32_t w[BITS];
-            const uint8_t *pp = p_tiles + s * P_STAGE_BYTES + p_off;
+            const uint32_t pp = p_base + (uint32_t)s * P_STAGE_BYTES;
 #pragma unroll
-            for (int i = 0; i < BITS; ++i) w[i] = *reinterpret_cast<const uint32_t *>(pp + i * P_PLANE_BYTES);
+            for (int i = 0; i < BITS; ++i)
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[i]) : "r"(pp + i * P_PLANE_BYTES) : "memory");
             uint32_t out[16];
             dequant_word<BITS>(w, T, out);
-            uint8_t *row = b_tiles + s * B_STAGE_BYTES + row_off;
+            const uint32_t row = b_base + (uint32_t)s * B_STAGE_BYTES;
 #pragma unroll
             for (int cj = 0; cj < 4; ++cj) {
                 const uint32_t chunk = ((uint32_t)(4 * v + cj)) ^ xr;
-                *reinterpret_cast<uint4 *>(row + chunk * 16) =
-                    make_uint4(out[4 * cj], out[4 * cj + 1], out[4 * cj + 2], out[4 * cj + 3]);
+                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(row + chunk * 16u), "r"(out[4 * cj]),
+                             "r"(out[4 * cj + 1]), "r"(out[4 * cj + 2]), "r"(out[4 * cj + 3]) : "memory");
             }
             fence_proxy_async_smem();
             __syncwarp();
