@@ -16,6 +16,7 @@
  *     W is logically [K x N]:  w[k][n] = s[k/group][n] * (q[k][n] - z[k/group][n])
  *     (paper Sec. 2.2, "Dequantization-based low-bit inference"), q and z unsigned integers
  *     in [0, 2^bits).
+ *   - Alignment: packed and workspace 256 bytes, x and y 16 bytes (else TMAN_ERR_SHAPE).
  *   - Legal shapes: bits in {1,2,3,4} for pack/unpack, {2,3,4} for the matmuls;
  *     group in {32,64,128}; K % 128 == 0; N % 8 == 0.  Anything else: TMAN_ERR_SHAPE /
  *     TMAN_ERR_UNSUPPORTED.
@@ -64,7 +65,8 @@ tman_status tman_packed_bytes(int K, int N, int bits, int group, size_t *out_byt
 tman_status tman_workspace_bytes(int op, int M, int K, int N, int bits, int group,
                                  size_t *out_bytes /*host*/);
 
-/* Zero a workspace (status word and split-K arrival counters). */
+/* Prepare a workspace: status word zero, partial-sum area marked "no sum pending".  After a call
+ * reported TMAN_ERR_TIMEOUT the workspace must be prepared again. */
 tman_status tman_workspace_init(void *workspace, size_t ws_bytes, tman_stream_t stream);
 
 /* Copy the workspace's status word to *out_status (host) and wait for `stream`. */

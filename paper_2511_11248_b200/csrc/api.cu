@@ -55,9 +55,8 @@ tman_status tman_workspace_init(void *workspace, size_t ws_bytes, tman_stream_t 
 {
     if (!workspace) return TMAN_ERR_NULL;
     if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
-    if (cudaMemsetAsync(workspace, 0, ws_bytes, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
-        return TMAN_ERR_CUDA;
-    return TMAN_OK;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return TMAN_ERR_SHAPE;
+    return launch_workspace_init(workspace, ws_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
 tman_status tman_read_status(const void *workspace, int *out_status, tman_stream_t stream)
@@ -117,7 +116,9 @@ tman_status tman_mpgemv(const void *packed, size_t packed_bytes, const void *x_f
     tman_status st = check_matmul(packed, packed_bytes, x_f16, y_f16, M, K, N, bits, group, workspace);
     if (st != TMAN_OK) return st;
     if (M > 8) return TMAN_ERR_SHAPE;
-    if (reinterpret_cast<uintptr_t>(x_f16) & 15) return TMAN_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(x_f16) & 15) || (reinterpret_cast<uintptr_t>(y_f16) & 15) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return TMAN_ERR_SHAPE;
     if (ws_bytes < mpgemv_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
     return launch_mpgemv(packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
                          reinterpret_cast<cudaStream_t>(stream));

@@ -55,12 +55,9 @@ __device__ inline bool header_matches(const void *packed, int K, int N, int bits
 }
 
 // ---- workspace ---------------------------------------------------------------------------
-// [0, 256)              status word (u32) + padding
-// [256, 256 + ctr)      split-K arrival counters (u32), zero between calls
-// [256 + ctr, ...)      fp32 split-K partial sums
+// [0, 256)      status word (u32) + padding
+// [256, ...)     fp32 split-K partial sums; "no sum pending" sentinel between calls
 constexpr size_t kWsStatusBytes = 256;
-
-__host__ __device__ inline size_t ws_counter_bytes(int N) { return up256((size_t)(N / 4) * 4); }
 
 // ---- argument checks (host) --------------------------------------------------------------
 inline tman_status check_format(int K, int N, int bits, int group)
@@ -112,7 +109,7 @@ tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int
                                  uint32_t *status, cudaStream_t s);
 tman_status launch_debug_luts(const void *x, int M, int K, float *lut, cudaStream_t s);
 size_t      mpgemv_workspace_bytes(int M, int K, int N);
-size_t      mpgemv_workspace_zero_prefix(int N);
+tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s);
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s);
 size_t      mpgemm_workspace_bytes(int M, int K, int N);

@@ -11,74 +11,74 @@
 // what allows 8-bit indices (two of the paper's 4-bit indices fused: one lookup covers eight
 // weights of one bit-plane).
 //
-// Per lane and column: sum_i 2^i * sum_{4 groups} T[group][index byte]  (shift-accumulate),
-// minus zero-point times the lane's activation sum, times the block scale (a lane's 32
-// activations never straddle a quantization block since group >= 32); the per-lane partials of
-// a column are then reduced across the lanes of the K-slice with warp shuffles, and K-slices
-// are combined through fp32 partial sums in the workspace: the last slice to arrive (a counter
-// per column group) adds them in slice order and writes fp16.
+// Per lane and column: sum_i 2^i * sum_{4 groups} T[group][index byte]  (shift-accumulate).
+// Lanes whose words share a quantization block are added first (one shuffle stage), then the
+// zero-point times the block's activation sum is subtracted and the block scale applied, then the
+// remaining lanes of the K-slice are reduced with a transposing shuffle reduction.  K-slices are
+// combined through fp32 partial sums in the workspace.  The partial-sum area holds a sentinel bit
+// pattern (a NaN no arithmetic produces) wherever no sum is pending; once its lookups are done,
+// every CTA polls the sums of its share of the output columns until none of them is the sentinel,
+// adds them in a fixed order, writes fp16 and puts the sentinel back.  The data are their own
+// "ready" flag, so no fence and no counter sits between the last lookup and the output; the poll
+// is bounded and reports TMAN_ERR_TIMEOUT.
+//
+// Streaming.  A warp works through small units (a few strips of four columns) and keeps the next
+// unit's plane words in a second set of registers, so that HBM reads overlap the lookups.  The
+// first loads are issued before the kernel waits for the previous kernel in the stream
+// (programmatic dependent launch): weights are constant input and the host has checked that
+// every read derived from (K, N, bits, group) is in bounds.
 #include "common.cuh"
 
 namespace tman {
-
-// Optional phase time stamps for experiments (compiled out of the library build).
-#ifdef TMAN_PHASE_TIMERS
-__device__ unsigned long long *tman_stamp_buf;
-#define TMAN_STAMP(i)                                                              \
-    do {                                                                           \
-        if (threadIdx.x == 0) {                                                    \
-            unsigned long long t_;                                                 \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                 \
-            tman_stamp_buf[blockIdx.x * 16 + (i)] = t_;                            \
-            tman_stamp_buf[blockIdx.x * 16 + 8 + (i)] = (unsigned long long)clock64(); \
-        }                                                                          \
-    } while (0)
-#else
-#define TMAN_STAMP(i) do {} while (0)
-#endif
 
 constexpr int kGemvThreads = 512;
 constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kGemvTableBytes = 128 * 1024;   // 4 groups x 256 entries x 32 slots x 4 B
 
+// "No sum pending": a NaN bit pattern that no floating-point operation returns.
+constexpr uint32_t kGemvSentinel = 0x7FA5A5A5u;
+constexpr uint32_t kGemvPollLimit = 1u << 21;  // polls of ~0.5 us each: about a second
+
 struct GemvParams {
     const uint8_t  *packed;
-    const uint32_t *planes;
-    const __half   *scales;
-    const uint16_t *zeros;
-    const __half   *x;        // first row of this launch
-    __half         *y;        // first row of this launch
+    const uint4    *planes;     // one uint4 = one plane word of the four columns of a strip
+    const uint2    *scales;     // four fp16 scales of a strip and block
+    const uint16_t *zeros;      // four zero-point nibbles of a strip and block
+    const __half   *x;          // first row of this launch
+    __half         *y;          // first row of this launch
     float          *partials;
-    uint32_t       *counters;
     uint32_t       *status;
-    int M;                    // rows in this launch (<= MT)
+    int M;                      // rows in this launch (<= MT)
     int K, N, bits, group;
-    int nkappa;               // K-slices
-    int P;                    // CTAs per K-slice
-    int units;                // warp-units per K-slice
+    int nkappa;                 // K-slices
+    int P;                      // CTAs per K-slice
+    int units;                  // warp-units per K-slice
+    int group_shift;            // log2(group)
+    int nblk;                   // K / group
 };
 
-template <int N_, int MASK>
+// Transposing reduction over the lanes selected by MASK, 2*MASK, ..., below END: every stage
+// halves the number of values a lane keeps (or, once one is left, plainly adds).  `base` is the
+// logical index of vals[0].
+template <int N_, int MASK, int END>
 struct LaneReduce {
-    // Transpose-reduce N_ values across the lanes selected by MASK, MASK/2, ..., 1: every stage
-    // halves the number of values a lane keeps (or, once one is left, plainly adds).
     static __device__ __forceinline__ void run(float *vals, int v, int &base)
     {
-        if constexpr (MASK >= 1) {
+        if constexpr (MASK < END) {
             if constexpr (N_ >= 2) {
                 constexpr int H = N_ / 2;
                 const bool up = (v & MASK) != 0;
 #pragma unroll
                 for (int j = 0; j < H; ++j) {
-                    float keep = up ? vals[j + H] : vals[j];
-                    float send = up ? vals[j] : vals[j + H];
+                    const float keep = up ? vals[j + H] : vals[j];
+                    const float send = up ? vals[j] : vals[j + H];
                     vals[j] = keep + __shfl_xor_sync(0xffffffffu, send, MASK);
                 }
                 base += up ? H : 0;
-                LaneReduce<H, MASK / 2>::run(vals, v, base);
+                LaneReduce<H, MASK * 2, END>::run(vals, v, base);
             } else {
                 vals[0] += __shfl_xor_sync(0xffffffffu, vals[0], MASK);
-                LaneReduce<1, MASK / 2>::run(vals, v, base);
+                LaneReduce<1, MASK * 2, END>::run(vals, v, base);
             }
         }
     }
@@ -98,28 +98,52 @@ __device__ __forceinline__ void load_rows(const uint8_t *p, float (&out)[MT])
     else { out[0] = t.x; out[1] = t.y; out[2] = t.z; out[3] = t.w; }
 }
 
+__device__ __forceinline__ float4 ld_volatile_f4(const float4 *p)
+{
+    float4 v;
+    asm volatile("ld.volatile.global.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ bool has_sentinel(const float4 &v)
+{
+    return __float_as_uint(v.x) == kGemvSentinel || __float_as_uint(v.y) == kGemvSentinel ||
+           __float_as_uint(v.z) == kGemvSentinel || __float_as_uint(v.w) == kGemvSentinel;
+}
+
 // byte offset of table entry (group c of the lane's word, index p, slot) inside the table area
 __device__ __forceinline__ constexpr uint32_t table_imm(int c) { return (uint32_t)(c >> 1) * 65536u + (uint32_t)(c & 1) * 128u; }
 
-template <int BITS, int MT, int S>
+// One unit's worth of a lane's inputs: its plane word of S strips, and the strips' scales and
+// zero-points of the lane's quantization block.
+template <int BITS, int S>
+struct UnitRegs {
+    uint4    w[S][BITS];
+    uint2    sc[S];
+    uint32_t z[S];
+};
+
+// BITS planes, MT rows per table entry, S strips per warp-unit and sub-warp, PRE = 1 when the
+// lanes v and v^1 share a quantization block (group >= 64): they are added before scaling.
+template <int BITS, int MT, int S, int PRE>
 __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     constexpr int W = 32 / MT;            // plane words (lanes) per K-slice
     constexpr int V = 4 * S * MT;         // values a lane produces per warp-unit
+    constexpr int V1 = PRE ? V / 2 : V;   // values it still holds when scales are applied
     constexpr int NKEEP = (V >= W) ? V / W : 1;
 
-    TMAN_STAMP(0);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int kappa = blockIdx.x / p.P, j = blockIdx.x % p.P;
-    const int words_total = p.K / 32;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int kappa = blockIdx.y, j = blockIdx.x;
+    const int words_total = p.K >> 5;
     const int word0 = kappa * W;
     const int nwords = min(W, words_total - word0);
     const int sub = lane / W, v = lane % W;
     const bool active = v < nwords;
-    const int nstrips = p.N / 4;
-    const int nblk = p.K / p.group;
-    const int B = active ? ((word0 + v) * 32) / p.group : 0;
+    const int nstrips = p.N >> 2;
+    const int nblk = p.nblk;
+    const int B = ((word0 + (active ? v : 0)) * 32) >> p.group_shift;
 
     // Let the next kernel in the stream start its own weight streaming while this one drains
     // (programmatic dependent launch); the header words are requested now and checked later.
@@ -128,37 +152,36 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
     for (int q = 0; q < 8; ++q) hdr[q] = __ldg(reinterpret_cast<const uint32_t *>(p.packed) + q);
 
-    uint4    wreg[S][BITS];
-    uint2    sreg[S];
-    uint32_t zreg[S];
-
-    auto load_unit = [&](int wu) {
+    // Loads are unconditional: a unit past the last one re-reads the last unit, a strip past the
+    // last one re-reads the last strip, a lane past the end of a ragged last slice re-reads word 0
+    // (its tables are all zero); none of those results is ever written.
+    const uint8_t *pw = reinterpret_cast<const uint8_t *>(p.planes + word0 + (active ? v : 0));
+    const uint2 *psc = p.scales + B;
+    const uint16_t *pz = p.zeros + B;
+    const uint32_t row_bytes = (uint32_t)words_total * 16u;      // one plane of one strip
+    const uint32_t strip_bytes = row_bytes * BITS;
+    auto load_unit = [&](UnitRegs<BITS, S> &r, int wu) {
+        const int u = min(wu, p.units - 1);
 #pragma unroll
         for (int s = 0; s < S; ++s) {
-            const int nb = (wu * MT + sub) * S + s;
-            const bool ok = active && nb < nstrips;
+            const uint32_t nb = (uint32_t)min((u * MT + sub) * S + s, nstrips - 1);
+            const uint8_t *q = pw + (size_t)nb * strip_bytes;
 #pragma unroll
             for (int i = 0; i < BITS; ++i) {
-                wreg[s][i] = make_uint4(0u, 0u, 0u, 0u);
-                if (ok)
-                    wreg[s][i] = __ldcs(reinterpret_cast<const uint4 *>(p.planes) +
-                                        ((size_t)nb * BITS + i) * words_total + word0 + v);
+                r.w[s][i] = __ldcs(reinterpret_cast<const uint4 *>(q));
+                q += row_bytes;
             }
-            sreg[s] = make_uint2(0u, 0u);
-            zreg[s] = 0u;
-            if (ok) {
-                sreg[s] = __ldg(reinterpret_cast<const uint2 *>(p.scales) + (size_t)nb * nblk + B);
-                zreg[s] = __ldg(p.zeros + (size_t)nb * nblk + B);
-            }
+            r.sc[s] = __ldg(psc + (size_t)nb * (uint32_t)nblk);
+            r.z[s] = __ldg(pz + (size_t)nb * (uint32_t)nblk);
         }
     };
 
     // Issue the first unit's weight loads before anything else: the packed buffer is constant
     // input and packed_bytes was checked on the host, so these reads are in bounds whatever the
     // header says.  Their latency overlaps the table build.
-    int wu = j + p.P * warp;
-    if (wu < p.units) load_unit(wu);
-    TMAN_STAMP(1);
+    const int wu0 = j + p.P * warp, wstride = p.P * kGemvWarps;
+    UnitRegs<BITS, S> regs[2];
+    load_unit(regs[0], wu0);
 
     // Everything below may depend on the previous kernel in the stream (activations, workspace).
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -174,7 +197,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
         for (int c = 0; c < 4; ++c) xraw[c] = __ldg(px + c);
     }
-    TMAN_STAMP(2);
+    load_unit(regs[1], wu0 + wstride);
 
     // ---- phase A: activation tables (paper Sec. 2.2; one table per 8 activations, 256 entries,
     // entry = 16-entry table of the low four + sum of the selected high four) -----------------
@@ -205,7 +228,6 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         }
     }
     __syncthreads();
-    TMAN_STAMP(3);
 
     // header check (uniform over the grid): a mismatch leaves every output untouched
     {
@@ -213,12 +235,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                             (hdr[3] == (uint32_t)p.K) && (hdr[4] == (uint32_t)p.N) &&
                             (hdr[5] == (uint32_t)p.bits) && (hdr[6] == (uint32_t)p.group) && (hdr[7] == 4u);
         if (!hdr_ok) {
-            if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
+            if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
             return;
         }
     }
 
-    // the lane's activation sum over its 32 activations (all-ones entries), for the zero-point term
+    // the activation sum of the lane's 32 activations (all-ones entries), for the zero-point term;
+    // with PRE, of the two lanes that share the block
     const uint32_t sub_off = (uint32_t)(v * MT * 4);
     float ssum[MT];
     {
@@ -231,20 +254,17 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
             for (int m = 0; m < MT; ++m) ssum[m] += t[m];
         }
+        if constexpr (PRE) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m) ssum[m] += __shfl_xor_sync(0xffffffffu, ssum[m], 1);
+        }
     }
 
-    bool first = true;
-    for (; wu < p.units; wu += p.P * kGemvWarps) {
-        if (!first) load_unit(wu);
-        first = false;
-
-        // ---- phase B: lookups, shift-accumulate, scale and zero-point (paper Sec. 4.3) --------
+    // ---- phase B: lookups, shift-accumulate, scale and zero-point (paper Sec. 4.3) --------------
+    auto compute_unit = [&](const UnitRegs<BITS, S> &r, int wu) {
         float vals[V];
 #pragma unroll
-        for (int s = 0; s < S; ++s) {
-            const __half2 s01 = *reinterpret_cast<const __half2 *>(&sreg[s].x);
-            const __half2 s23 = *reinterpret_cast<const __half2 *>(&sreg[s].y);
-            const float sc[4] = {__low2float(s01), __high2float(s01), __low2float(s23), __high2float(s23)};
+        for (int s = 0; s < S; ++s)
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
                 float a[MT];
@@ -252,8 +272,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 for (int m = 0; m < MT; ++m) a[m] = 0.f;
 #pragma unroll
                 for (int i = 0; i < BITS; ++i) {
-                    const uint32_t w = (c4 == 0) ? wreg[s][i].x : (c4 == 1) ? wreg[s][i].y
-                                     : (c4 == 2) ? wreg[s][i].z : wreg[s][i].w;
+                    const uint32_t w = (c4 == 0) ? r.w[s][i].x : (c4 == 1) ? r.w[s][i].y
+                                     : (c4 == 2) ? r.w[s][i].z : r.w[s][i].w;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         // byte 1 <- index byte c of the word, byte 0 <- the lane's slot offset
@@ -264,71 +284,138 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                         for (int m = 0; m < MT; ++m) a[m] = fmaf(t[m], (float)(1 << i), a[m]);
                     }
                 }
-                const float zf = (float)((zreg[s] >> (4 * c4)) & 0xFu);
 #pragma unroll
-                for (int m = 0; m < MT; ++m)
-                    vals[(s * 4 + c4) * MT + m] = sc[c4] * fmaf(-zf, ssum[m], a[m]);
+                for (int m = 0; m < MT; ++m) vals[(s * 4 + c4) * MT + m] = a[m];
             }
-        }
 
-        TMAN_STAMP(4);
-        // ---- reduce the K-slice's lanes (warp shuffles) -----------------------------------------
+        // lanes v and v^1 hold the two words of one block: add them first, keeping half the columns
         int base = 0;
-        LaneReduce<V, W / 2>::run(vals, v, base);
-        const bool writer = (V >= W) ? true : ((v & (W / V - 1)) == 0);
-        const int col0 = (wu * MT + sub) * S * 4;      // first column of this sub-warp's strips
-        TMAN_STAMP(5);
-
-        if (p.nkappa == 1) {
-            if (writer) {
+        LaneReduce<V, 1, PRE ? 2 : 1>::run(vals, v, base);
+        const bool up = PRE && (v & 1);
+        // scales and zero-points of the columns this lane still holds
+        if constexpr (S >= 2 || !PRE) {
+            constexpr int S1 = PRE ? S / 2 : S;
 #pragma unroll
-                for (int e = 0; e < NKEEP; ++e) {
-                    const int idx = base + e, m = idx % MT, n = col0 + idx / MT;
-                    if (n < p.N && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(vals[e]);
+            for (int s = 0; s < S1; ++s) {
+                const uint2 scq = up ? r.sc[s + (PRE ? S1 : 0)] : r.sc[s];
+                const uint32_t zq = up ? r.z[s + (PRE ? S1 : 0)] : r.z[s];
+                const __half2 s01 = *reinterpret_cast<const __half2 *>(&scq.x);
+                const __half2 s23 = *reinterpret_cast<const __half2 *>(&scq.y);
+                const float sc[4] = {__low2float(s01), __high2float(s01), __low2float(s23), __high2float(s23)};
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    const float zf = (float)((zq >> (4 * c4)) & 0xFu);
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) {
+                        float &val = vals[(s * 4 + c4) * MT + m];
+                        val = sc[c4] * fmaf(-zf, ssum[m], val);
+                    }
                 }
             }
         } else {
-            if (writer) {
+            // one strip, two of its four columns left
+            const uint32_t scq = up ? r.sc[0].y : r.sc[0].x;
+            const uint32_t zq = up ? (r.z[0] >> 8) : r.z[0];
+            const __half2 s01 = *reinterpret_cast<const __half2 *>(&scq);
+            const float sc[2] = {__low2float(s01), __high2float(s01)};
 #pragma unroll
-                for (int e = 0; e < NKEEP; ++e) {
-                    const int idx = base + e, m = idx % MT, n = col0 + idx / MT;
-                    if (n < p.N) p.partials[((size_t)kappa * MT + m) * p.N + n] = vals[e];
+            for (int c2 = 0; c2 < 2; ++c2) {
+                const float zf = (float)((zq >> (4 * c2)) & 0xFu);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    float &val = vals[c2 * MT + m];
+                    val = sc[c2] * fmaf(-zf, ssum[m], val);
                 }
-            }
-            // ---- combine K-slices: the last slice to arrive sums them in slice order ------------
-            __threadfence();
-            __syncwarp();
-            uint32_t old = 0;
-            if (lane == 0) old = atomicAdd(p.counters + wu, 1u);
-            old = __shfl_sync(0xffffffffu, old, 0);
-            TMAN_STAMP(6);
-            if (old == (uint32_t)(p.nkappa - 1)) {
-                __threadfence();
-                constexpr int C = 4 * S * MT;           // columns of the warp-unit
-                const int cw0 = wu * C;
-                for (int idx = lane; idx < MT * C; idx += 32) {
-                    const int m = idx / C, n = cw0 + idx % C;
-                    if (n < p.N && m < p.M) {
-                        float acc = 0.f;
-                        for (int kp = 0; kp < p.nkappa; ++kp)
-                            acc += __ldcg(p.partials + ((size_t)kp * MT + m) * p.N + n);
-                        p.y[(size_t)m * p.N + n] = __float2half_rn(acc);
-                    }
-                }
-                if (lane == 0) p.counters[wu] = 0u;
             }
         }
+        // the other lanes of the K-slice
+        LaneReduce<V1, PRE ? 2 : 1, W>::run(vals, v, base);
+        const bool writer = (V >= W) ? true : (v < V);
+        const int col0 = (wu * MT + sub) * S * 4;      // first column of this sub-warp's strips
+        if (writer) {
+#pragma unroll
+            for (int e = 0; e < NKEEP; ++e) {
+                const int idx = base + e, m = idx % MT, n = col0 + idx / MT;
+                if (n < p.N && m < p.M) {
+                    if (p.nkappa == 1) p.y[(size_t)m * p.N + n] = __float2half_rn(vals[e]);
+                    else p.partials[((size_t)kappa * MT + m) * p.N + n] = vals[e];
+                }
+            }
+        }
+    };
+
+    for (int wu = wu0; wu < p.units; wu += 2 * wstride) {
+        compute_unit(regs[0], wu);
+        load_unit(regs[0], wu + 2 * wstride);
+        if (wu + wstride >= p.units) break;            // uniform over the warp
+        compute_unit(regs[1], wu + wstride);
+        load_unit(regs[1], wu + 3 * wstride);
     }
-    TMAN_STAMP(7);
+
+    // ---- combine K-slices: every CTA polls the partial sums of its share of the columns ----------
+    if (p.nkappa > 1) {
+        const int cta = blockIdx.y * gridDim.x + blockIdx.x, G = gridDim.x * gridDim.y;
+        const int ng = p.N >> 2;
+        const int g_lo = (int)(((long long)ng * cta) / G), g_hi = (int)(((long long)ng * (cta + 1)) / G);
+        const int col_lo = g_lo * 4;
+        const int ngrp = g_hi - g_lo;
+        const int items = ngrp * p.M;                       // one item = four columns of one row
+        const size_t stride4 = (size_t)MT * p.N / 4;
+        // SP adjacent lanes share an item and split the slices among them (slice kp goes to lane
+        // kp % SP); their sums are added in a fixed order, so the result does not depend on timing
+        int SP = 1;
+        while (SP < 8 && 2 * SP <= p.nkappa && items * 2 * SP <= kGemvThreads) SP *= 2;
+        const int part = tid & (SP - 1);
+        const float sv = __uint_as_float(kGemvSentinel);
+        bool gave_up = false;
+        for (int item0 = 0; item0 < items; item0 += kGemvThreads / SP) {
+            const int item = item0 + tid / SP;
+            const bool alive = item < items;
+            const int m = alive ? item / ngrp : 0, n = col_lo + 4 * (alive ? item % ngrp : 0);
+            float4 *src = reinterpret_cast<float4 *>(p.partials + (size_t)m * p.N + n);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int kp = part; alive && kp < p.nkappa; kp += 4 * SP) {
+                float4 t[4];
+                bool ready = false;
+                for (uint32_t tries = 0; !ready && tries < kGemvPollLimit; ++tries) {
+                    ready = true;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (kp + q * SP < p.nkappa) t[q] = ld_volatile_f4(src + (size_t)(kp + q * SP) * stride4);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (kp + q * SP < p.nkappa) ready = ready && !has_sentinel(t[q]);
+                }
+                if (!ready) { gave_up = true; break; }
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (kp + q * SP < p.nkappa) {
+                        acc.x += t[q].x; acc.y += t[q].y; acc.z += t[q].z; acc.w += t[q].w;
+                        src[(size_t)(kp + q * SP) * stride4] = make_float4(sv, sv, sv, sv);
+                    }
+            }
+            for (int mask = 1; mask < SP; mask <<= 1) {
+                acc.x += __shfl_xor_sync(0xffffffffu, acc.x, mask);
+                acc.y += __shfl_xor_sync(0xffffffffu, acc.y, mask);
+                acc.z += __shfl_xor_sync(0xffffffffu, acc.z, mask);
+                acc.w += __shfl_xor_sync(0xffffffffu, acc.w, mask);
+            }
+            gave_up = __any_sync(0xffffffffu, gave_up);
+            if (alive && part == 0 && !gave_up) {
+                const __half2 h01 = __floats2half2_rn(acc.x, acc.y), h23 = __floats2half2_rn(acc.z, acc.w);
+                uint2 o;
+                o.x = *reinterpret_cast<const uint32_t *>(&h01);
+                o.y = *reinterpret_cast<const uint32_t *>(&h23);
+                *reinterpret_cast<uint2 *>(p.y + (size_t)m * p.N + n) = o;
+            }
+        }
+        if (gave_up) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
+    }
 }
 
-template <int BITS, int MT>
-static constexpr int strips_per_unit() { return (BITS == 2 ? 8 : 4) / MT; }
-
-template <int BITS, int MT>
+template <int BITS, int MT, int S, int PRE>
 static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
 {
-    constexpr int S = strips_per_unit<BITS, MT>();
     constexpr int W = 32 / MT;
     const int words_total = p.K / 32;
     p.nkappa = (words_total + W - 1) / W;
@@ -337,11 +424,13 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     const int nstrips = p.N / 4;
     p.units = (nstrips + S * MT - 1) / (S * MT);
     if (p.P > p.units) p.P = p.units;
-    auto kern = mpgemv_kernel<BITS, MT, S>;
+    // every CTA must be resident while it polls for the others' partial sums
+    if ((long long)p.nkappa * p.P > (long long)sms) return TMAN_ERR_UNSUPPORTED;
+    auto kern = mpgemv_kernel<BITS, MT, S, PRE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvTableBytes) != cudaSuccess)
         return TMAN_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(p.nkappa * p.P));
+    cfg.gridDim = dim3((unsigned)p.P, (unsigned)p.nkappa);
     cfg.blockDim = dim3(kGemvThreads);
     cfg.dynamicSmemBytes = kGemvTableBytes;
     cfg.stream = s;
@@ -354,13 +443,36 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     return TMAN_OK;
 }
 
+// strips per unit: small enough that two units fit in registers, large enough for V >= 4
+template <int BITS, int MT, int PRE>
+static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
+{
+    constexpr int S = (MT == 1) ? ((BITS == 2) ? 2 : 1) : 1;
+    return launch_one<BITS, MT, S, PRE>(p, sms, s);
+}
+
 template <int BITS>
 static tman_status launch_rows(GemvParams p, int rows, int sms, cudaStream_t s)
 {
     p.M = rows;
-    if (rows == 1) return launch_one<BITS, 1>(p, sms, s);
-    if (rows == 2) return launch_one<BITS, 2>(p, sms, s);
-    return launch_one<BITS, 4>(p, sms, s);
+    const bool pre = p.group >= 64;
+    if (rows == 1) return pre ? launch_mt<BITS, 1, 1>(p, sms, s) : launch_mt<BITS, 1, 0>(p, sms, s);
+    if (rows == 2) return pre ? launch_mt<BITS, 2, 1>(p, sms, s) : launch_mt<BITS, 2, 0>(p, sms, s);
+    return pre ? launch_mt<BITS, 4, 1>(p, sms, s) : launch_mt<BITS, 4, 0>(p, sms, s);
+}
+
+__global__ void ws_fill_kernel(uint32_t *ws, size_t words)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < words) ws[i] = (i < kWsStatusBytes / 4) ? 0u : kGemvSentinel;
+}
+
+// status word (and its padding) zero, everything after it "no sum pending"
+tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s)
+{
+    const size_t words = ws_bytes / 4;
+    ws_fill_kernel<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(static_cast<uint32_t *>(ws), words);
+    return launch_status();
 }
 
 size_t mpgemv_workspace_bytes(int M, int K, int N)
@@ -368,11 +480,8 @@ size_t mpgemv_workspace_bytes(int M, int K, int N)
     (void)M;
     // worst case: rows are processed four at a time with K-slices of 8 plane words
     const size_t nkappa = (size_t)(K / 32 + 7) / 8;
-    return kWsStatusBytes + ws_counter_bytes(N) + nkappa * 4 * (size_t)N * sizeof(float);
+    return kWsStatusBytes + nkappa * 4 * (size_t)N * sizeof(float);
 }
-
-// bytes at the start of a workspace that must be zero before a call (status word and counters)
-size_t mpgemv_workspace_zero_prefix(int N) { return kWsStatusBytes + ws_counter_bytes(N); }
 
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s)
@@ -385,14 +494,15 @@ tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int
     uint8_t *w8 = static_cast<uint8_t *>(ws);
     GemvParams p;
     p.packed = pk;
-    p.planes = reinterpret_cast<const uint32_t *>(pk + L.planes_off);
-    p.scales = reinterpret_cast<const __half *>(pk + L.scales_off);
+    p.planes = reinterpret_cast<const uint4 *>(pk + L.planes_off);
+    p.scales = reinterpret_cast<const uint2 *>(pk + L.scales_off);
     p.zeros = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
     p.status = reinterpret_cast<uint32_t *>(w8);
-    p.counters = reinterpret_cast<uint32_t *>(w8 + kWsStatusBytes);
-    p.partials = reinterpret_cast<float *>(w8 + kWsStatusBytes + ws_counter_bytes(N));
+    p.partials = reinterpret_cast<float *>(w8 + kWsStatusBytes);
     p.K = K; p.N = N; p.bits = bits; p.group = group;
     p.M = 0; p.nkappa = 0; p.P = 0; p.units = 0;
+    p.group_shift = (group == 32) ? 5 : (group == 64) ? 6 : 7;
+    p.nblk = K / group;
     // rows go through in batches of at most four (a table entry carries up to four rows)
     for (int m0 = 0; m0 < M; m0 += 4) {
         const int rows = (M - m0 < 4) ? (M - m0) : 4;

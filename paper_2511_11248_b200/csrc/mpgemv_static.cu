@@ -4,8 +4,8 @@
 // matmul: an inference runtime that sizes one arena at start-up and forbids cudaMalloc afterwards
 // (an allocation can synchronise the device and breaks a latency budget), a plug-in that runs inside
 // another framework's stream callback, code between "begin" and "end" of a region where the
-// allocator is locked.  tman_mpgemv needs scratch memory (a status word, arrival counters and
-// the fp32 partial sums of the K-slices) that such a caller has nowhere to put.  Here that
+// allocator is locked.  tman_mpgemv needs scratch memory (a status word and the fp32
+// partial sums of the K-slices) that such a caller has nowhere to put.  Here that
 // scratch is a fixed array that is part of the library image: every GPU that loads the library
 // holds kStaticWsBytes of it from load until the process exits, and nothing is allocated at
 // call time.
@@ -58,7 +58,9 @@ extern "C" tman_status tman_mpgemv_static(const void *packed, size_t packed_byte
     if (packed_bytes < make_layout(K, N, bits, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
     if (bits < 2) return TMAN_ERR_UNSUPPORTED;
     if (M < 1 || M > 8) return TMAN_ERR_SHAPE;
-    if ((reinterpret_cast<uintptr_t>(packed) & 255) || (reinterpret_cast<uintptr_t>(x_f16) & 15)) return TMAN_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(packed) & 255) || (reinterpret_cast<uintptr_t>(x_f16) & 15) ||
+        (reinterpret_cast<uintptr_t>(y_f16) & 15))
+        return TMAN_ERR_SHAPE;
     // the fixed array is the whole budget: a shape whose scratch does not fit is refused
     const size_t need = mpgemv_workspace_bytes(M, K, N);
     if (need > kStaticWsBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
@@ -67,9 +69,10 @@ extern "C" tman_status tman_mpgemv_static(const void *packed, size_t packed_byte
     st = static_ws(&ws);
     if (st != TMAN_OK) return st;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    // The array keeps whatever the last call left.  The status word and the arrival counters
-    // must start at zero; the partial sums are written before they are read.
-    if (cudaMemsetAsync(ws, 0, mpgemv_workspace_zero_prefix(N), s) != cudaSuccess) return TMAN_ERR_CUDA;
+    // The array keeps whatever the last call left.  The status word must start at zero and the
+    // partial-sum area must say "no sum pending" everywhere this call will look.
+    st = launch_workspace_init(ws, need, s);
+    if (st != TMAN_OK) return st;
     st = launch_mpgemv(packed, x_f16, y_f16, M, K, N, bits, group, ws, kStaticWsBytes, s);
     if (st != TMAN_OK) return st;
     if (status_dev &&
