@@ -114,6 +114,27 @@ __device__ __forceinline__ bool has_sentinel(const float4 &v)
 // byte offset of table entry (group c of the lane's word, index p, slot) inside the table area
 __device__ __forceinline__ constexpr uint32_t table_imm(int c) { return (uint32_t)(c >> 1) * 65536u + (uint32_t)(c & 1) * 128u; }
 
+// The tables start at the first byte of dynamic shared memory.  The kernel has no static shared
+// memory, so that byte sits right after the per-CTA reserved region, at shared-window address
+// kGemvSmemBase (the host checks cudaDevAttrReservedSharedMemoryPerBlock, the kernel checks its
+// own base).  A lookup can then use the byte-permute result (index byte << 8 | slot offset) as
+// the address register, with the table's offset folded into the instruction's immediate: no add
+// per lookup.
+constexpr uint32_t kGemvSmemBase = 1024;
+
+template <int MT, uint32_t IMM>
+__device__ __forceinline__ void lookup_rows(uint32_t off, float (&out)[MT])
+{
+    if constexpr (MT == 1) {
+        asm volatile("ld.shared.f32 %0, [%1 + %2];" : "=f"(out[0]) : "r"(off), "n"(IMM));
+    } else if constexpr (MT == 2) {
+        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2 + %3];" : "=f"(out[0]), "=f"(out[1]) : "r"(off), "n"(IMM));
+    } else {
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4 + %5];"
+                     : "=f"(out[0]), "=f"(out[1]), "=f"(out[2]), "=f"(out[3]) : "r"(off), "n"(IMM));
+    }
+}
+
 // One unit's worth of a lane's inputs: its plane word of S strips, and the strips' scales and
 // zero-points of the lane's quantization block.
 template <int BITS, int S>
@@ -234,7 +255,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         const bool hdr_ok = (hdr[0] == 0x4E414D54u) && (hdr[1] == 0x30303242u) && (hdr[2] == kVersion) &&
                             (hdr[3] == (uint32_t)p.K) && (hdr[4] == (uint32_t)p.N) &&
                             (hdr[5] == (uint32_t)p.bits) && (hdr[6] == (uint32_t)p.group) && (hdr[7] == 4u);
-        if (!hdr_ok) {
+        if (!hdr_ok || (uint32_t)__cvta_generic_to_shared(smem) != kGemvSmemBase) {
             if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
             return;
         }
@@ -274,15 +295,16 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 for (int i = 0; i < BITS; ++i) {
                     const uint32_t w = (c4 == 0) ? r.w[s][i].x : (c4 == 1) ? r.w[s][i].y
                                      : (c4 == 2) ? r.w[s][i].z : r.w[s][i].w;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        // byte 1 <- index byte c of the word, byte 0 <- the lane's slot offset
-                        const uint32_t off = __byte_perm(w, sub_off, 0x7604u | ((uint32_t)c << 4));
-                        float t[MT];
-                        load_rows<MT>(smem + table_imm(c) + off, t);
-#pragma unroll
-                        for (int m = 0; m < MT; ++m) a[m] = fmaf(t[m], (float)(1 << i), a[m]);
-                    }
+                    // byte 1 <- index byte c of the word, byte 0 <- the lane's slot offset
+#define TMAN_LOOKUP(c)                                                                          \
+    {                                                                                           \
+        const uint32_t off = __byte_perm(w, sub_off, 0x7604u | ((uint32_t)(c) << 4));           \
+        float t[MT];                                                                            \
+        lookup_rows<MT, kGemvSmemBase + table_imm(c)>(off, t);                                  \
+        _Pragma("unroll") for (int m = 0; m < MT; ++m) a[m] = fmaf(t[m], (float)(1 << i), a[m]); \
+    }
+                    TMAN_LOOKUP(0) TMAN_LOOKUP(1) TMAN_LOOKUP(2) TMAN_LOOKUP(3)
+#undef TMAN_LOOKUP
                 }
 #pragma unroll
                 for (int m = 0; m < MT; ++m) vals[(s * 4 + c4) * MT + m] = a[m];
@@ -426,6 +448,11 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     if (p.P > p.units) p.P = p.units;
     // every CTA must be resident while it polls for the others' partial sums
     if ((long long)p.nkappa * p.P > (long long)sms) return TMAN_ERR_UNSUPPORTED;
+    int dev = 0, reserved = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev) != cudaSuccess)
+        return TMAN_ERR_CUDA;
+    if ((uint32_t)reserved != kGemvSmemBase) return TMAN_ERR_UNSUPPORTED;
     auto kern = mpgemv_kernel<BITS, MT, S, PRE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvTableBytes) != cudaSuccess)
         return TMAN_ERR_CUDA;
