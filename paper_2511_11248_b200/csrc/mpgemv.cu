@@ -146,11 +146,18 @@ struct UnitRegs {
 
 // BITS planes, MT rows per table entry, S strips per warp-unit and sub-warp, PRE = 1 when the
 // lanes v and v^1 share a quantization block (group >= 64): they are added before scaling.
-template <int BITS, int MT, int S, int PRE>
+// HALF (MT = 1 only): K-slices of 16 plane words instead of 32, i.e. 64 KB of tables that cost
+// half as much to build.  The two half-warps then work on different strips and read the same 64
+// tables; entry rows hold all 64 slots (slot = word + 16 * index byte) and the second half-warp
+// visits the index bytes of a word in the order 1,0,3,2, so that the 32 lanes still address 32
+// different banks.
+template <int BITS, int MT, int S, int PRE, int HALF>
 __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    constexpr int W = 32 / MT;            // plane words (lanes) per K-slice
+    static_assert(!HALF || MT == 1, "half slices are for single-row tables");
+    constexpr int W = HALF ? 16 : 32 / MT; // plane words (lanes) per K-slice
+    constexpr int SUBS = 32 / W;           // sub-warps, each on its own strips
     constexpr int V = 4 * S * MT;         // values a lane produces per warp-unit
     constexpr int V1 = PRE ? V / 2 : V;   // values it still holds when scales are applied
     constexpr int NKEEP = (V >= W) ? V / W : 1;
@@ -185,7 +192,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         const int u = min(wu, p.units - 1);
 #pragma unroll
         for (int s = 0; s < S; ++s) {
-            const uint32_t nb = (uint32_t)min((u * MT + sub) * S + s, nstrips - 1);
+            const uint32_t nb = (uint32_t)min((u * SUBS + sub) * S + s, nstrips - 1);
             const uint8_t *q = pw + (size_t)nb * strip_bytes;
 #pragma unroll
             for (int i = 0; i < BITS; ++i) {
@@ -207,45 +214,76 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     // Everything below may depend on the previous kernel in the stream (activations, workspace).
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // The activations of this thread's table slot (one plane word = 32 activations of one row).
-    const int vb = lane / MT, mb = lane % MT;
-    const bool live = (vb < nwords) && (mb < p.M);
-    uint4 xraw[4];
+    if constexpr (HALF) {
+        // thread (slot, chunk): slot = word + 16 * index byte of the table it fills, chunk = the
+        // three high index bits of its 32 entries
+        const int slot = tid & 63, chunk = tid >> 6;
+        const int gv = slot & 15, gc = slot >> 4;
+        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+        if (gv < nwords) raw = __ldg(reinterpret_cast<const uint4 *>(p.x + (size_t)(word0 + gv) * 32 + gc * 8));
+        load_unit(regs[1], wu0 + wstride);
+        float xv[8];
+        const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) xraw[c] = make_uint4(0u, 0u, 0u, 0u);
-    if (live) {
-        const uint4 *px = reinterpret_cast<const uint4 *>(p.x + (size_t)mb * p.K + (size_t)(word0 + vb) * 32);
+        for (int q = 0; q < 4; ++q) {
+            const float2 f = __half22float2(h2[q]);
+            xv[2 * q] = f.x;
+            xv[2 * q + 1] = f.y;
+        }
+        float lo[16];
+        lut16(xv[0], xv[1], xv[2], xv[3], lo);
+        float hi = 0.f;
+        if (chunk & 1) hi += xv[5];
+        if (chunk & 2) hi += xv[6];
+        if (chunk & 4) hi += xv[7];
+        uint8_t *dst = smem + (uint32_t)(chunk * 32) * 256u + (uint32_t)slot * 4u;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) xraw[c] = __ldg(px + c);
-    }
-    load_unit(regs[1], wu0 + wstride);
+        for (int q = 0; q < 2; ++q) {
+            const float base = q ? hi + xv[4] : hi;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) *reinterpret_cast<float *>(dst + (q * 16 + e) * 256) = lo[e] + base;
+        }
+    } else {
+        // The activations of this thread's table slot (one plane word = 32 activations of one row).
+        const int vb = lane / MT, mb = lane % MT;
+        const bool live = (vb < nwords) && (mb < p.M);
+        uint4 xraw[4];
+    #pragma unroll
+        for (int c = 0; c < 4; ++c) xraw[c] = make_uint4(0u, 0u, 0u, 0u);
+        if (live) {
+            const uint4 *px = reinterpret_cast<const uint4 *>(p.x + (size_t)mb * p.K + (size_t)(word0 + vb) * 32);
+    #pragma unroll
+            for (int c = 0; c < 4; ++c) xraw[c] = __ldg(px + c);
+        }
+        load_unit(regs[1], wu0 + wstride);
 
-    // ---- phase A: activation tables (paper Sec. 2.2; one table per 8 activations, 256 entries,
-    // entry = 16-entry table of the low four + sum of the selected high four) -----------------
-    {
-        // warp w fills the entries whose high index nibble is w, for all four groups of the word
-        const int ph = warp;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            float xv[8];
-            const __half2 *h2 = reinterpret_cast<const __half2 *>(&xraw[c]);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float2 f = __half22float2(h2[q]);
-                xv[2 * q] = f.x;
-                xv[2 * q + 1] = f.y;
+        // ---- phase A: activation tables (paper Sec. 2.2; one table per 8 activations, 256 entries,
+        // entry = 16-entry table of the low four + sum of the selected high four) -----------------
+        {
+            // warp w fills the entries whose high index nibble is w, for all four groups of the word
+            const int ph = warp;
+    #pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float xv[8];
+                const __half2 *h2 = reinterpret_cast<const __half2 *>(&xraw[c]);
+    #pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float2 f = __half22float2(h2[q]);
+                    xv[2 * q] = f.x;
+                    xv[2 * q + 1] = f.y;
+                }
+                float lo[16];
+                lut16(xv[0], xv[1], xv[2], xv[3], lo);
+                float hi = 0.f;
+                if (ph & 1) hi += xv[4];
+                if (ph & 2) hi += xv[5];
+                if (ph & 4) hi += xv[6];
+                if (ph & 8) hi += xv[7];
+                uint8_t *dst = smem + table_imm(c) + (uint32_t)(ph * 16) * 256u + (uint32_t)lane * 4u;
+    #pragma unroll
+                for (int pl = 0; pl < 16; ++pl)
+                    *reinterpret_cast<float *>(dst + pl * 256) = lo[pl] + hi;
             }
-            float lo[16];
-            lut16(xv[0], xv[1], xv[2], xv[3], lo);
-            float hi = 0.f;
-            if (ph & 1) hi += xv[4];
-            if (ph & 2) hi += xv[5];
-            if (ph & 4) hi += xv[6];
-            if (ph & 8) hi += xv[7];
-            uint8_t *dst = smem + table_imm(c) + (uint32_t)(ph * 16) * 256u + (uint32_t)lane * 4u;
-#pragma unroll
-            for (int pl = 0; pl < 16; ++pl)
-                *reinterpret_cast<float *>(dst + pl * 256) = lo[pl] + hi;
         }
     }
     __syncthreads();
@@ -264,6 +302,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     // the activation sum of the lane's 32 activations (all-ones entries), for the zero-point term;
     // with PRE, of the two lanes that share the block
     const uint32_t sub_off = (uint32_t)(v * MT * 4);
+    // HALF: slot offset inside a row = (v + 16 * byte) * 4; the byte visited at step jj is jj for
+    // the first half-warp and jj ^ 1 for the second, so 64 * (jj & ~1) goes into the immediate and
+    // the rest (0 or 64) into one of two registers
+    const uint32_t off_even = (uint32_t)(v * 4 + 64 * sub), off_odd = (uint32_t)(v * 4 + 64 * (1 - sub));
+    uint32_t sel_h[4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) sel_h[jj] = 0x7604u | ((uint32_t)(jj ^ sub) << 4);
     float ssum[MT];
     {
 #pragma unroll
@@ -271,7 +316,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             float t[MT];
-            load_rows<MT>(smem + table_imm(c) + 255u * 256u + sub_off, t);
+            if constexpr (HALF) load_rows<MT>(smem + 255u * 256u + (uint32_t)(v + 16 * c) * 4u, t);
+            else load_rows<MT>(smem + table_imm(c) + 255u * 256u + sub_off, t);
 #pragma unroll
             for (int m = 0; m < MT; ++m) ssum[m] += t[m];
         }
@@ -298,9 +344,14 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                     // byte 1 <- index byte c of the word, byte 0 <- the lane's slot offset
 #define TMAN_LOOKUP(c)                                                                          \
     {                                                                                           \
-        const uint32_t off = __byte_perm(w, sub_off, 0x7604u | ((uint32_t)(c) << 4));           \
         float t[MT];                                                                            \
-        lookup_rows<MT, kGemvSmemBase + table_imm(c)>(off, t);                                  \
+        if constexpr (HALF) {                                                                   \
+            const uint32_t off = __byte_perm(w, ((c) & 1) ? off_odd : off_even, sel_h[c]);      \
+            lookup_rows<MT, kGemvSmemBase + 64u * ((c) & ~1)>(off, t);                          \
+        } else {                                                                                \
+            const uint32_t off = __byte_perm(w, sub_off, 0x7604u | ((uint32_t)(c) << 4));       \
+            lookup_rows<MT, kGemvSmemBase + table_imm(c)>(off, t);                              \
+        }                                                                                       \
         _Pragma("unroll") for (int m = 0; m < MT; ++m) a[m] = fmaf(t[m], (float)(1 << i), a[m]); \
     }
                     TMAN_LOOKUP(0) TMAN_LOOKUP(1) TMAN_LOOKUP(2) TMAN_LOOKUP(3)
@@ -353,7 +404,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         // the other lanes of the K-slice
         LaneReduce<V1, PRE ? 2 : 1, W>::run(vals, v, base);
         const bool writer = (V >= W) ? true : (v < V);
-        const int col0 = (wu * MT + sub) * S * 4;      // first column of this sub-warp's strips
+        const int col0 = (wu * SUBS + sub) * S * 4;    // first column of this sub-warp's strips
         if (writer) {
 #pragma unroll
             for (int e = 0; e < NKEEP; ++e) {
@@ -435,16 +486,18 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     }
 }
 
-template <int BITS, int MT, int S, int PRE>
+template <int BITS, int MT, int S, int PRE, int HALF>
 static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
 {
-    constexpr int W = 32 / MT;
+    constexpr int W = HALF ? 16 : 32 / MT;
+    constexpr int SUBS = 32 / W;
+    constexpr int kSmem = HALF ? kGemvTableBytes / 2 : kGemvTableBytes;
     const int words_total = p.K / 32;
     p.nkappa = (words_total + W - 1) / W;
     p.P = sms / p.nkappa;
     if (p.P < 1) p.P = 1;
     const int nstrips = p.N / 4;
-    p.units = (nstrips + S * MT - 1) / (S * MT);
+    p.units = (nstrips + S * SUBS - 1) / (S * SUBS);
     if (p.P > p.units) p.P = p.units;
     // every CTA must be resident while it polls for the others' partial sums
     if ((long long)p.nkappa * p.P > (long long)sms) return TMAN_ERR_UNSUPPORTED;
@@ -453,13 +506,13 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
         cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev) != cudaSuccess)
         return TMAN_ERR_CUDA;
     if ((uint32_t)reserved != kGemvSmemBase) return TMAN_ERR_UNSUPPORTED;
-    auto kern = mpgemv_kernel<BITS, MT, S, PRE>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvTableBytes) != cudaSuccess)
+    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
         return TMAN_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.P, (unsigned)p.nkappa);
     cfg.blockDim = dim3(kGemvThreads);
-    cfg.dynamicSmemBytes = kGemvTableBytes;
+    cfg.dynamicSmemBytes = kSmem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -475,7 +528,7 @@ template <int BITS, int MT, int PRE>
 static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
 {
     constexpr int S = (MT == 1) ? ((BITS == 2) ? 2 : 1) : 1;
-    return launch_one<BITS, MT, S, PRE>(p, sms, s);
+    return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0>(p, sms, s);
 }
 
 template <int BITS>
