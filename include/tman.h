@@ -111,6 +111,17 @@ tman_status tman_mpgemv(const void *packed, size_t packed_bytes, const void *x_f
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream);
 
+/* Decode for `count` (1..4) weight matrices that read the same activations, in one launch (paper
+ * Sec. 5 "Implementation", graph optimisation: the table precomputation is shared by the
+ * projections with a common input, e.g. Q/K/V or gate/up).  All matrices have the same K, bits and
+ * group; matrix g has N[g] output columns and its own packed buffer and output y_f16[g]
+ * ([M][N[g]], fp16).  packed, packed_bytes, y_f16 and N are HOST arrays of `count` entries (read
+ * during the call); their entries follow the rules of tman_mpgemv.  The workspace must hold
+ * tman_workspace_bytes(0, M, K, N[0] + ... + N[count-1], bits, group). */
+tman_status tman_mpgemv_grouped(int count, const void *const *packed /*host*/, const size_t *packed_bytes /*host*/,
+                                const void *x_f16, void *const *y_f16 /*host*/, int M, int K, const int *N /*host*/,
+                                int bits, int group, void *workspace, size_t ws_bytes, tman_stream_t stream);
+
 /* Prefill (paper Sec. 4.1 two-level LUT dequantization, Fig. 7; Sec. 4.2 three-stage pipeline,
  * Fig. 9): packed tiles are staged in shared memory, rebuilt into fp16 tiles through the
  * repack step and the per-(block, column) conversion table, and multiplied on the tensor

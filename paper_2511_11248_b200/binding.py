@@ -22,7 +22,7 @@ OP_GEMV, OP_GEMM, OP_AUX = 0, 1, 2
 EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
-    "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_mpgemv_static",
+    "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_mpgemv_static", "tman_mpgemv_grouped",
 ]
 
 _lib = None
@@ -56,6 +56,7 @@ def lib() -> C.CDLL:
         L.tman_mpgemv.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, sz, vp]
         L.tman_mpgemm.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, sz, vp]
         L.tman_mpgemv_static.argtypes = [vp, sz, vp, vp, i, i, i, i, i, vp, vp]
+        L.tman_mpgemv_grouped.argtypes = [i, C.POINTER(vp), C.POINTER(sz), vp, C.POINTER(vp), i, i, C.POINTER(i), i, i, vp, sz, vp]
         L.tman_debug_indices.argtypes = [vp, i, i, i, i, vp, vp, sz, vp]
         L.tman_debug_luts.argtypes = [vp, i, i, vp, vp]
         for name in EXPORTS[2:]:
@@ -136,6 +137,18 @@ def tman_mpgemv_static(packed, x, y, M, K, N, bits, group, status=None, stream=N
     _check(lib().tman_mpgemv_static(_ptr(packed), packed.numel() * packed.element_size(), _ptr(x), _ptr(y),
                                     M, K, N, bits, group, _ptr(status), _stream(stream)),
            "tman_mpgemv_static")
+
+
+def tman_mpgemv_grouped(packed_list, x, y_list, M, K, N_list, bits, group, workspace, stream=None) -> None:
+    """Decode for several weight matrices that share the activations x, in one launch."""
+    n = len(packed_list)
+    pk = (C.c_void_p * n)(*[_ptr(t) for t in packed_list])
+    pb = (C.c_size_t * n)(*[t.numel() * t.element_size() for t in packed_list])
+    ys = (C.c_void_p * n)(*[_ptr(t) for t in y_list])
+    ns = (C.c_int * n)(*[int(v) for v in N_list])
+    _check(lib().tman_mpgemv_grouped(n, pk, pb, _ptr(x), ys, M, K, ns, bits, group, _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream)),
+           "tman_mpgemv_grouped")
 
 
 def tman_mpgemm(packed, x, y, M, K, N, bits, group, workspace, stream=None) -> None:

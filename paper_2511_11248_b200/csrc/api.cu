@@ -124,6 +124,26 @@ tman_status tman_mpgemv(const void *packed, size_t packed_bytes, const void *x_f
                          reinterpret_cast<cudaStream_t>(stream));
 }
 
+tman_status tman_mpgemv_grouped(int count, const void *const *packed, const size_t *packed_bytes,
+                                const void *x_f16, void *const *y_f16, int M, int K, const int *N,
+                                int bits, int group, void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    if (!packed || !packed_bytes || !y_f16 || !N) return TMAN_ERR_NULL;
+    if (count < 1 || count > 4) return TMAN_ERR_SHAPE;
+    long long ntot = 0;
+    for (int g = 0; g < count; ++g) {
+        tman_status st = check_matmul(packed[g], packed_bytes[g], x_f16, y_f16[g], M, K, N[g], bits, group, workspace);
+        if (st != TMAN_OK) return st;
+        if (reinterpret_cast<uintptr_t>(y_f16[g]) & 15) return TMAN_ERR_SHAPE;
+        ntot += N[g];
+    }
+    if (M > 8 || ntot > (1 << 30)) return TMAN_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(x_f16) & 15) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return TMAN_ERR_SHAPE;
+    if (ws_bytes < mpgemv_workspace_bytes(M, K, (int)ntot)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_mpgemv_grouped(count, packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
+                                 reinterpret_cast<cudaStream_t>(stream));
+}
+
 tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream)

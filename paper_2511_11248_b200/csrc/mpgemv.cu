@@ -39,17 +39,26 @@ constexpr int kGemvTableBytes = 128 * 1024;   // 4 groups x 256 entries x 32 slo
 constexpr uint32_t kGemvSentinel = 0x7FA5A5A5u;
 constexpr uint32_t kGemvPollLimit = 1u << 21;  // polls of ~0.5 us each: about a second
 
+// Up to kGemvMaxGroup weight matrices that share the activations (same K, bits, group) go through
+// one launch: their output columns are concatenated, the tables are built once (paper Sec. 5:
+// one table precomputation shared by the projections that read the same input).
+constexpr int kGemvMaxGroup = 4;
+
 struct GemvParams {
-    const uint8_t  *packed;
-    const uint4    *planes;     // one uint4 = one plane word of the four columns of a strip
-    const uint2    *scales;     // four fp16 scales of a strip and block
-    const uint16_t *zeros;      // four zero-point nibbles of a strip and block
+    const uint8_t  *packed[kGemvMaxGroup];
+    const uint4    *planes[kGemvMaxGroup];   // one uint4 = one plane word of the four columns of a strip
+    const uint2    *scales[kGemvMaxGroup];   // four fp16 scales of a strip and block
+    const uint16_t *zeros[kGemvMaxGroup];    // four zero-point nibbles of a strip and block
+    __half         *y[kGemvMaxGroup];        // first row of this launch
+    int Ng[kGemvMaxGroup];                   // output columns of each matrix
+    int unit0[kGemvMaxGroup];                // first warp-unit of each matrix
+    int col0[kGemvMaxGroup];                 // first concatenated column of each matrix
+    int count;                               // matrices in this launch
     const __half   *x;          // first row of this launch
-    __half         *y;          // first row of this launch
     float          *partials;
     uint32_t       *status;
     int M;                      // rows in this launch (<= MT)
-    int K, N, bits, group;
+    int K, N, bits, group;      // N = total (concatenated) columns
     int nkappa;                 // K-slices
     int P;                      // CTAs per K-slice
     int units;                  // warp-units per K-slice
@@ -142,6 +151,8 @@ struct UnitRegs {
     uint4    w[S][BITS];
     uint2    sc[S];
     uint32_t z[S];
+    int      g;        // matrix of the unit
+    int      col;      // concatenated column of the lane's first strip
 };
 
 // BITS planes, MT rows per table entry, S strips per warp-unit and sub-warp, PRE = 1 when the
@@ -169,30 +180,50 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     const int nwords = min(W, words_total - word0);
     const int sub = lane / W, v = lane % W;
     const bool active = v < nwords;
-    const int nstrips = p.N >> 2;
     const int nblk = p.nblk;
     const int B = ((word0 + (active ? v : 0)) * 32) >> p.group_shift;
 
     // Let the next kernel in the stream start its own weight streaming while this one drains
     // (programmatic dependent launch); the header words are requested now and checked later.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    uint32_t hdr[8];
+    bool hdr_ok = true;
+    {
+        uint32_t hdr[kGemvMaxGroup][8];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) hdr[q] = __ldg(reinterpret_cast<const uint32_t *>(p.packed) + q);
+        for (int g = 0; g < kGemvMaxGroup; ++g)
+            if (g < p.count) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) hdr[g][q] = __ldg(reinterpret_cast<const uint32_t *>(p.packed[g]) + q);
+            }
+#pragma unroll
+        for (int g = 0; g < kGemvMaxGroup; ++g)
+            if (g < p.count)
+                hdr_ok = hdr_ok && (hdr[g][0] == 0x4E414D54u) && (hdr[g][1] == 0x30303242u) && (hdr[g][2] == kVersion) &&
+                         (hdr[g][3] == (uint32_t)p.K) && (hdr[g][4] == (uint32_t)p.Ng[g]) &&
+                         (hdr[g][5] == (uint32_t)p.bits) && (hdr[g][6] == (uint32_t)p.group) && (hdr[g][7] == 4u);
+    }
 
     // Loads are unconditional: a unit past the last one re-reads the last unit, a strip past the
     // last one re-reads the last strip, a lane past the end of a ragged last slice re-reads word 0
     // (its tables are all zero); none of those results is ever written.
-    const uint8_t *pw = reinterpret_cast<const uint8_t *>(p.planes + word0 + (active ? v : 0));
-    const uint2 *psc = p.scales + B;
-    const uint16_t *pz = p.zeros + B;
+    const uint32_t lane_word = (uint32_t)(word0 + (active ? v : 0));
     const uint32_t row_bytes = (uint32_t)words_total * 16u;      // one plane of one strip
     const uint32_t strip_bytes = row_bytes * BITS;
     auto load_unit = [&](UnitRegs<BITS, S> &r, int wu) {
         const int u = min(wu, p.units - 1);
+        int g = 0;
+#pragma unroll
+        for (int t = 1; t < kGemvMaxGroup; ++t) g += (t < p.count && u >= p.unit0[t]) ? 1 : 0;
+        const int lu = u - p.unit0[g];
+        const int nstrips = p.Ng[g] >> 2;
+        const uint8_t *pw = reinterpret_cast<const uint8_t *>(p.planes[g] + lane_word);
+        const uint2 *psc = p.scales[g] + B;
+        const uint16_t *pz = p.zeros[g] + B;
+        r.g = g;
+        r.col = p.col0[g] + (lu * SUBS + sub) * S * 4;
 #pragma unroll
         for (int s = 0; s < S; ++s) {
-            const uint32_t nb = (uint32_t)min((u * SUBS + sub) * S + s, nstrips - 1);
+            const uint32_t nb = (uint32_t)min((lu * SUBS + sub) * S + s, nstrips - 1);
             const uint8_t *q = pw + (size_t)nb * strip_bytes;
 #pragma unroll
             for (int i = 0; i < BITS; ++i) {
@@ -289,14 +320,9 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     __syncthreads();
 
     // header check (uniform over the grid): a mismatch leaves every output untouched
-    {
-        const bool hdr_ok = (hdr[0] == 0x4E414D54u) && (hdr[1] == 0x30303242u) && (hdr[2] == kVersion) &&
-                            (hdr[3] == (uint32_t)p.K) && (hdr[4] == (uint32_t)p.N) &&
-                            (hdr[5] == (uint32_t)p.bits) && (hdr[6] == (uint32_t)p.group) && (hdr[7] == 4u);
-        if (!hdr_ok || (uint32_t)__cvta_generic_to_shared(smem) != kGemvSmemBase) {
-            if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
-            return;
-        }
+    if (!hdr_ok || (uint32_t)__cvta_generic_to_shared(smem) != kGemvSmemBase) {
+        if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
+        return;
     }
 
     // the activation sum of the lane's 32 activations (all-ones entries), for the zero-point term;
@@ -404,13 +430,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         // the other lanes of the K-slice
         LaneReduce<V1, PRE ? 2 : 1, W>::run(vals, v, base);
         const bool writer = (V >= W) ? true : (v < V);
-        const int col0 = (wu * SUBS + sub) * S * 4;    // first column of this sub-warp's strips
-        if (writer) {
+        if (writer && wu < p.units) {
+            const int lim = p.col0[r.g] + p.Ng[r.g];   // end of this matrix's columns
 #pragma unroll
             for (int e = 0; e < NKEEP; ++e) {
-                const int idx = base + e, m = idx % MT, n = col0 + idx / MT;
-                if (n < p.N && m < p.M) {
-                    if (p.nkappa == 1) p.y[(size_t)m * p.N + n] = __float2half_rn(vals[e]);
+                const int idx = base + e, m = idx % MT, n = r.col + idx / MT;
+                if (n < lim && m < p.M) {
+                    if (p.nkappa == 1) p.y[r.g][(size_t)m * p.Ng[r.g] + (n - p.col0[r.g])] = __float2half_rn(vals[e]);
                     else p.partials[((size_t)kappa * MT + m) * p.N + n] = vals[e];
                 }
             }
@@ -479,7 +505,10 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 uint2 o;
                 o.x = *reinterpret_cast<const uint32_t *>(&h01);
                 o.y = *reinterpret_cast<const uint32_t *>(&h23);
-                *reinterpret_cast<uint2 *>(p.y + (size_t)m * p.N + n) = o;
+                int g = 0;
+#pragma unroll
+                for (int t = 1; t < kGemvMaxGroup; ++t) g += (t < p.count && n >= p.col0[t]) ? 1 : 0;
+                *reinterpret_cast<uint2 *>(p.y[g] + (size_t)m * p.Ng[g] + (n - p.col0[g])) = o;
             }
         }
         if (gave_up) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
@@ -496,8 +525,12 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     p.nkappa = (words_total + W - 1) / W;
     p.P = sms / p.nkappa;
     if (p.P < 1) p.P = 1;
-    const int nstrips = p.N / 4;
-    p.units = (nstrips + S * SUBS - 1) / (S * SUBS);
+    p.units = 0;
+    for (int g = 0; g < p.count; ++g) {
+        p.unit0[g] = p.units;
+        p.units += (p.Ng[g] / 4 + S * SUBS - 1) / (S * SUBS);
+    }
+    for (int g = p.count; g < kGemvMaxGroup; ++g) p.unit0[g] = p.units;
     if (p.P > p.units) p.P = p.units;
     // every CTA must be resident while it polls for the others' partial sums
     if ((long long)p.nkappa * p.P > (long long)sms) return TMAN_ERR_UNSUPPORTED;
@@ -563,23 +596,32 @@ size_t mpgemv_workspace_bytes(int M, int K, int N)
     return kWsStatusBytes + nkappa * 4 * (size_t)N * sizeof(float);
 }
 
-tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
-                          int group, void *ws, size_t ws_bytes, cudaStream_t s)
+tman_status launch_mpgemv_grouped(int count, const void *const *packed, const void *x, void *const *y, int M, int K,
+                                  const int *Ns, int bits, int group, void *ws, size_t ws_bytes, cudaStream_t s)
 {
     (void)ws_bytes;
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
-    Layout L = make_layout(K, N, bits, group);
-    const uint8_t *pk = static_cast<const uint8_t *>(packed);
     uint8_t *w8 = static_cast<uint8_t *>(ws);
     GemvParams p;
-    p.packed = pk;
-    p.planes = reinterpret_cast<const uint4 *>(pk + L.planes_off);
-    p.scales = reinterpret_cast<const uint2 *>(pk + L.scales_off);
-    p.zeros = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
+    p.count = count;
+    p.N = 0;
+    for (int g = 0; g < kGemvMaxGroup; ++g) {
+        const int gg = g < count ? g : 0;
+        Layout L = make_layout(K, Ns[gg], bits, group);
+        const uint8_t *pk = static_cast<const uint8_t *>(packed[gg]);
+        p.packed[g] = pk;
+        p.planes[g] = reinterpret_cast<const uint4 *>(pk + L.planes_off);
+        p.scales[g] = reinterpret_cast<const uint2 *>(pk + L.scales_off);
+        p.zeros[g] = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
+        p.Ng[g] = g < count ? Ns[g] : 0;
+        p.col0[g] = p.N;
+        p.unit0[g] = 0;
+        if (g < count) p.N += Ns[g];
+    }
     p.status = reinterpret_cast<uint32_t *>(w8);
     p.partials = reinterpret_cast<float *>(w8 + kWsStatusBytes);
-    p.K = K; p.N = N; p.bits = bits; p.group = group;
+    p.K = K; p.bits = bits; p.group = group;
     p.M = 0; p.nkappa = 0; p.P = 0; p.units = 0;
     p.group_shift = (group == 32) ? 5 : (group == 64) ? 6 : 7;
     p.nblk = K / group;
@@ -587,7 +629,8 @@ tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int
     for (int m0 = 0; m0 < M; m0 += 4) {
         const int rows = (M - m0 < 4) ? (M - m0) : 4;
         p.x = static_cast<const __half *>(x) + (size_t)m0 * K;
-        p.y = static_cast<__half *>(y) + (size_t)m0 * N;
+        for (int g = 0; g < kGemvMaxGroup; ++g)
+            p.y[g] = static_cast<__half *>(y[g < count ? g : 0]) + (size_t)m0 * p.Ng[g];
         tman_status st;
         if (bits == 2) st = launch_rows<2>(p, rows, sms, s);
         else if (bits == 3) st = launch_rows<3>(p, rows, sms, s);
@@ -595,6 +638,12 @@ tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int
         if (st != TMAN_OK) return st;
     }
     return TMAN_OK;
+}
+
+tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
+                          int group, void *ws, size_t ws_bytes, cudaStream_t s)
+{
+    return launch_mpgemv_grouped(1, &packed, x, &y, M, K, &N, bits, group, ws, ws_bytes, s);
 }
 
 }  // namespace tman
