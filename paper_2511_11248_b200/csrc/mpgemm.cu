@@ -30,8 +30,9 @@ constexpr int BM = 128, BN = 128, BK = 64;
 constexpr int NSTAGE = 4;
 constexpr int A_HALF_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
-constexpr int NUM_DEQ_WARPS = 8;
-constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS);
+constexpr int NUM_DEQ_WARPS = 8;                // warps that fill one weight tile
+constexpr int NUM_DEQ_GROUPS = 2;               // groups of such warps; they take turns, two k-blocks each
+constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS * NUM_DEQ_GROUPS);
 constexpr int P_PLANE_BYTES = (BN / 4) * (BK / 32) * 16;       // one plane of a packed tile: 32 strips x 2 words x 16 B
 constexpr int smem_bytes(int mh, int bits)
 {
@@ -363,7 +364,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // A warp owns 16 columns and both plane words of a k-block: lane = (strip of the warp, word,
         // column of the strip).  With this split the 32 lanes read 32 different banks of the staged
         // plane words and write eight different 16-byte bank groups per quarter-warp.
-        const int wd = warp - 2;
+        const int wd = (warp - 2) & (NUM_DEQ_WARPS - 1), grp = (warp - 2) / NUM_DEQ_WARPS;
         const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
         const int n_local = wd * 16 + sl * 4 + c;
         const int n = tile_n * BN + n_local;
@@ -378,7 +379,6 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
         const uint16_t *pz = p.zeros + (size_t)nb * nblk;
 
-        // scale and zero-point of the next quantization block are fetched one block ahead
         auto fetch_sz = [&](int B, __half &sv, uint32_t &zz) {
             sv = __float2half(0.f);
             zz = 0u;
@@ -388,20 +388,30 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             }
         };
         ConvTable<BITS> T;
-        int cur_B = -1;
-        const int B_step = (p.group == 32) ? 2 : 1;        // this lane's next block
-        __half sv_next;
-        uint32_t zz_next;
-        fetch_sz((v * 32) >> gshift, sv_next, zz_next);
+        int cur_B = -1, next_B = -1;
+        __half sv_next = __float2half(0.f);
+        uint32_t zz_next = 0u;
+        auto block_of = [&](int kb) { return ((2 * kb + v) * 32) >> gshift; };
+        // k-blocks of this group: 2*grp, 2*grp+1, 2*grp+2*NUM_DEQ_GROUPS, ...
+        auto next_kb = [&](int kb) { return (kb & 1) ? kb + 2 * NUM_DEQ_GROUPS - 1 : kb + 1; };
 
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb = 2 * grp; kb < num_kb; kb = next_kb(kb)) {
             const int s = kb % NSTAGE;
             const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
-            const int Bk = ((2 * kb + v) * 32) >> gshift;
+            const int Bk = block_of(kb);
             if (Bk != cur_B) {
+                if (next_B != Bk) fetch_sz(Bk, sv_next, zz_next);
                 cur_B = Bk;
                 T.build(sv_next, zz_next);
-                fetch_sz(Bk + B_step, sv_next, zz_next);
+            }
+            // scale and zero-point of the block after this one are fetched one k-block ahead
+            {
+                const int kn = next_kb(kb);
+                const int Bn = block_of(kn);
+                if (kn < num_kb && Bn != cur_B && Bn != next_B) {
+                    next_B = Bn;
+                    fetch_sz(Bn, sv_next, zz_next);
+                }
             }
             if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
             uint32_t w[BITS];
@@ -428,12 +438,11 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (ok) {
             tcgen05_fence_after();
             const int quarter = warp & 3;                 // tensor-memory lanes this warp may read
-            const int col_half = wd >> 2;                 // columns [0,64) or [64,128)
+            const int part = (warp - 2) >> 2;             // 32 of the tile's 128 columns
 #pragma unroll 1
-            for (int hc = 0; hc < 2 * MH; ++hc) {
-                const int h = hc >> 1, cc = hc & 1;
+            for (int h = 0; h < MH; ++h) {
                 const int m = tile_m * (BM * MH) + h * BM + quarter * 32 + lane;
-                const int col = col_half * 64 + cc * 32;
+                const int col = part * 32;
                 uint32_t r[32];
                 tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * BN + col), r);
                 tcgen05_wait_ld();
