@@ -2,19 +2,22 @@
 // (paper Sec. 4.1 "Unified Layout through Fused LUT-based Dequantization", Fig. 7;
 //  Sec. 4.2 "Pipelining to Hide Dequantization Overhead", Fig. 9).
 //
-// One CTA computes a 128 x 128 tile of y.  Three kinds of agents run concurrently on a ring of
+// A CTA computes tiles of 128*MH tokens x up to 128 output channels, one after the other (one CTA per
+// SM, each with an equal share of the output).  Four kinds of agents run concurrently on a ring of
 // shared-memory stages guarded by mbarriers (the paper's DMA / vector-core / matrix-core stages):
 //   * warp 0, one lane : TMA loads of the fp16 activation tile (128-byte swizzle) and of the packed
 //                        bit-plane words of the weight tile (one box per plane);
-//   * warps 2..9       : read the staged plane words of their column, rebuild the codes
+//   * warps 2..17      : (two groups of eight that take turns, two k-blocks each) read the staged
+//                        plane words of their column, rebuild the codes
 //                        (level 1: bit-serial -> bit-parallel), look every code up in the
 //                        per-(block, column) conversion table kept in registers and addressed
 //                        with byte-permute instructions (level 2: scale and zero-point baked in),
 //                        and write the fp16 weight tile in the K-major swizzled layout the
 //                        tensor core reads;
-//   * warp 1, one lane : tcgen05.mma (M128 N128 K16, fp16 x fp16 -> fp32 in tensor memory);
-//                        tcgen05.commit hands the stage back.
-// The dequantization warps then become the epilogue: tcgen05.ld, round to fp16, store.
+//   * warp 1, one lane : tcgen05.mma (M128 N<=128 K16, fp16 x fp16 -> fp32 in tensor memory), one
+//                        per row block; tcgen05.commit hands the stage back;
+//   * warps 18..21     : epilogue of the previous tile (tcgen05.ld, round to fp16, store) while the
+//                        next tile accumulates into the second set of tensor-memory columns.
 // Every wait is bounded: when a bound is hit the kernel records TMAN_ERR_TIMEOUT, stops issuing
 // work, and still reaches the common tear-down that frees tensor memory.
 #include "common.cuh"
@@ -32,7 +35,8 @@ constexpr int A_HALF_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_DEQ_WARPS = 8;                // warps that fill one weight tile
 constexpr int NUM_DEQ_GROUPS = 2;               // groups of such warps; they take turns, two k-blocks each
-constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS * NUM_DEQ_GROUPS);
+constexpr int NUM_EPI_WARPS = 4;                // one per quarter of the tensor-memory lanes
+constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS * NUM_DEQ_GROUPS + NUM_EPI_WARPS);
 constexpr int P_PLANE_BYTES = (BN / 4) * (BK / 32) * 16;       // one plane of a packed tile: 32 strips x 2 words x 16 B
 constexpr int smem_bytes(int mh, int bits)
 {
@@ -48,6 +52,8 @@ struct GemmParams {
     uint32_t       *status;
     int M, K, N, bits, group;
     int tiles_m, tiles_n;
+    int sms;
+    int R;          // column ranges per row tile
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -273,12 +279,47 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
         }
 }
 
+// Work of a CTA.  The output is cut into row tiles of 128*MH tokens and, inside a row tile, into R
+// column ranges of (almost) equal width, a multiple of 16 columns.  The tiles_m * R items are dealt
+// to the CTAs round-robin; a CTA walks through an item in sub-tiles of at most 128 columns, again of
+// (almost) equal width.  Every role derives the same list from (blockIdx, gridDim).
+struct SubTile { int tile_m, col0, bn; };
+
+struct TileWalk {
+    int item, nitems, stride, tiles_m, R, n16;
+    int tm, lo, len, nsub, j;
+    __device__ TileWalk(const GemmParams &p, int cta, int ncta)
+        : item(cta - ncta), nitems(p.tiles_m * p.R), stride(ncta), tiles_m(p.tiles_m), R(p.R),
+          n16((p.N + 15) >> 4),   // a last unit may reach 8 columns past N: computed, never stored
+          tm(0), lo(0), len(0), nsub(0), j(0) {}
+    __device__ bool next(SubTile &t)
+    {
+        if (j == nsub) {
+            item += stride;
+            if (item >= nitems) return false;
+            tm = item % tiles_m;
+            const int r = item / tiles_m;
+            lo = (int)(((long long)n16 * r) / R);
+            len = (int)(((long long)n16 * (r + 1)) / R) - lo;
+            nsub = (len + BN / 16 - 1) / (BN / 16);
+            j = 0;
+        }
+        const int u0 = lo + (len * j) / nsub, u1 = lo + (len * (j + 1)) / nsub;
+        t.tile_m = tm;
+        t.col0 = u0 * 16;
+        t.bn = (u1 - u0) * 16;
+        ++j;
+        return true;
+    }
+};
+
 template <int BITS, int MH>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const GemmParams p)
 {
     constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
-    constexpr int TMEM_COLS = MH * BN;                 // one fp32 accumulator of BN columns per row block
+    constexpr int ACC_COLS = MH * BN;                  // one fp32 accumulator of BN columns per row block
+    constexpr int TMEM_COLS = 2 * ACC_COLS;            // two sets: the epilogue of a sub-tile overlaps the next one
     constexpr int P_STAGE_BYTES = BITS * P_PLANE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {
@@ -291,16 +332,14 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     uint8_t *p_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + P_STAGE_BYTES));
     // bars[0..NSTAGE) loaded (TMA), [NSTAGE..2NSTAGE) full (dequantized), [2NSTAGE..3NSTAGE) empty,
-    // [3NSTAGE] accumulator ready
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * NSTAGE + 1);
-    uint32_t *fail_flag = tmem_slot + 1;
+    // then accumulator full[2], accumulator empty[2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * NSTAGE + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile_m = blockIdx.x % p.tiles_m, tile_n = blockIdx.x / p.tiles_m;
     const int num_kb = p.K / BK;
 
     const uint32_t loaded0 = smem_u32(bars), full0 = smem_u32(bars + NSTAGE), empty0 = smem_u32(bars + 2 * NSTAGE),
-                   accum_bar = smem_u32(bars + 3 * NSTAGE);
+                   accf0 = smem_u32(bars + 3 * NSTAGE), acce0 = smem_u32(bars + 3 * NSTAGE + 2);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NSTAGE; ++s) {
@@ -308,8 +347,10 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             mbar_init(full0 + 8 * s, NUM_DEQ_WARPS);
             mbar_init(empty0 + 8 * s, 1);
         }
-        mbar_init(accum_bar, 1);
-        *fail_flag = 0;
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(accf0 + 8 * b, 1);
+            mbar_init(acce0 + 8 * b, NUM_EPI_WARPS);
+        }
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -322,44 +363,56 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
 
     bool ok = true;
+    TileWalk walk(p, (int)blockIdx.x, (int)gridDim.x);
+    SubTile t;
     if (warp == 0) {
-        // ---- stage 1: activation tiles by TMA ------------------------------------------------
+        // ---- stage 1: activation tiles and packed weight tiles by TMA -------------------------
         if (lane == 0) {
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % NSTAGE;
-                const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
-                if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
-                mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + P_STAGE_BYTES);
-                tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, tile_m * (BM * MH), loaded0 + 8 * s);
+            uint32_t it = 0;
+            while (ok && walk.next(t)) {
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % NSTAGE);
+                    const uint32_t ph = (it / NSTAGE) & 1u;
+                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
+                    mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + P_STAGE_BYTES);
+                    tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, t.tile_m * (BM * MH), loaded0 + 8 * s);
 #pragma unroll
-                for (int i = 0; i < BITS; ++i)
-                    tma_load_3d(smem_u32(p_tiles + s * P_STAGE_BYTES + i * P_PLANE_BYTES), &tmap_w, kb * (BK / 8), i,
-                                tile_n * (BN / 4), loaded0 + 8 * s);
+                    for (int i = 0; i < BITS; ++i)
+                        tma_load_3d(smem_u32(p_tiles + s * P_STAGE_BYTES + i * P_PLANE_BYTES), &tmap_w, kb * (BK / 8), i,
+                                    t.col0 / 4, loaded0 + 8 * s);
+                }
             }
         }
     } else if (warp == 1) {
         // ---- stage 3: tensor-core MMA --------------------------------------------------------
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % NSTAGE;
-                const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
-                if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
+            uint32_t it = 0, ti = 0;
+            while (ok && walk.next(t)) {
+                const uint32_t buf = ti & 1u, aph = (ti >> 1) & 1u;
+                if (!mbar_wait(acce0 + 8 * buf, aph ^ 1u)) { ok = false; break; }
                 tcgen05_fence_after();
-                const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
+                const uint32_t idesc = (1u << 4) | ((uint32_t)(t.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % NSTAGE);
+                    const uint32_t ph = (it / NSTAGE) & 1u;
+                    if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
 #pragma unroll
-                for (int j = 0; j < BK / 16; ++j)
+                    for (int j = 0; j < BK / 16; ++j)
 #pragma unroll
-                    for (int h = 0; h < MH; ++h) {
-                        const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES + h * A_HALF_BYTES));
-                        tcgen05_mma_f16(tmem_base + (uint32_t)(h * BN), adesc + 2 * j, bdesc + 2 * j, idesc,
-                                        (kb > 0 || j > 0) ? 1u : 0u);
-                    }
-                tcgen05_commit(empty0 + 8 * s);
+                        for (int h = 0; h < MH; ++h) {
+                            const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES + h * A_HALF_BYTES));
+                            tcgen05_mma_f16(tmem_base + buf * ACC_COLS + (uint32_t)(h * BN), adesc + 2 * j, bdesc + 2 * j, idesc,
+                                            (kb > 0 || j > 0) ? 1u : 0u);
+                        }
+                    tcgen05_commit(empty0 + 8 * s);
+                }
+                if (ok) tcgen05_commit(accf0 + 8 * buf);
+                ++ti;
             }
-            if (ok) tcgen05_commit(accum_bar);
         }
-    } else {
+    } else if (warp < 2 + NUM_DEQ_WARPS * NUM_DEQ_GROUPS) {
         // ---- stage 2: two-level lookup dequantization ----------------------------------------
         // A warp owns 16 columns and both plane words of a k-block: lane = (strip of the warp, word,
         // column of the strip).  With this split the 32 lanes read 32 different banks of the staged
@@ -367,102 +420,116 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int wd = (warp - 2) & (NUM_DEQ_WARPS - 1), grp = (warp - 2) / NUM_DEQ_WARPS;
         const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
         const int n_local = wd * 16 + sl * 4 + c;
-        const int n = tile_n * BN + n_local;
-        const bool valid = n < p.N;
-        const int nb = n >> 2;
         const int nblk = p.K / p.group;
         const int gshift = (p.group == 32) ? 5 : (p.group == 64) ? 6 : 7;
         const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
         const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
         const uint32_t xr = (uint32_t)(n_local & 7);
         const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
-        const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
-        const uint16_t *pz = p.zeros + (size_t)nb * nblk;
-
-        auto fetch_sz = [&](int B, __half &sv, uint32_t &zz) {
-            sv = __float2half(0.f);
-            zz = 0u;
-            if (valid && B < nblk) {
-                sv = __ldg(ps + (size_t)B * 4);
-                zz = ((uint32_t)__ldg(pz + B) >> (4 * c)) & 0xFu;
-            }
-        };
-        ConvTable<BITS> T;
-        int cur_B = -1, next_B = -1;
-        __half sv_next = __float2half(0.f);
-        uint32_t zz_next = 0u;
         auto block_of = [&](int kb) { return ((2 * kb + v) * 32) >> gshift; };
-        // k-blocks of this group: 2*grp, 2*grp+1, 2*grp+2*NUM_DEQ_GROUPS, ...
+        // k-blocks of this group: 2*grp, 2*grp+1, 2*grp+2*NUM_DEQ_GROUPS, ... (num_kb is even)
         auto next_kb = [&](int kb) { return (kb & 1) ? kb + 2 * NUM_DEQ_GROUPS - 1 : kb + 1; };
 
-        for (int kb = 2 * grp; kb < num_kb; kb = next_kb(kb)) {
-            const int s = kb % NSTAGE;
-            const uint32_t ph = (uint32_t)(kb / NSTAGE) & 1u;
-            const int Bk = block_of(kb);
-            if (Bk != cur_B) {
-                if (next_B != Bk) fetch_sz(Bk, sv_next, zz_next);
-                cur_B = Bk;
-                T.build(sv_next, zz_next);
-            }
-            // scale and zero-point of the block after this one are fetched one k-block ahead
-            {
-                const int kn = next_kb(kb);
-                const int Bn = block_of(kn);
-                if (kn < num_kb && Bn != cur_B && Bn != next_B) {
-                    next_B = Bn;
-                    fetch_sz(Bn, sv_next, zz_next);
+        uint32_t it0 = 0;                                  // pipeline position of the sub-tile's first k-block
+        while (ok && walk.next(t)) {
+            const int n = t.col0 + n_local;
+            const bool valid = n_local < t.bn && n < p.N;   // columns past the sub-tile are not used by the MMA
+            const int nb = n >> 2;
+            const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
+            const uint16_t *pz = p.zeros + (size_t)nb * nblk;
+            auto fetch_sz = [&](int B, __half &sv, uint32_t &zz) {
+                sv = __float2half(0.f);
+                zz = 0u;
+                if (valid && B < nblk) {
+                    sv = __ldg(ps + (size_t)B * 4);
+                    zz = ((uint32_t)__ldg(pz + B) >> (4 * c)) & 0xFu;
                 }
-            }
-            if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
-            uint32_t w[BITS];
-            const uint32_t pp = p_base + (uint32_t)s * P_STAGE_BYTES;
-#pragma unroll
-            for (int i = 0; i < BITS; ++i)
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[i]) : "r"(pp + i * P_PLANE_BYTES) : "memory");
-            uint32_t out[16];
-            dequant_word<BITS>(w, T, out);
-            const uint32_t row = b_base + (uint32_t)s * B_STAGE_BYTES;
-#pragma unroll
-            for (int cj = 0; cj < 4; ++cj) {
-                const uint32_t chunk = ((uint32_t)(4 * v + cj)) ^ xr;
-                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(row + chunk * 16u), "r"(out[4 * cj]),
-                             "r"(out[4 * cj + 1]), "r"(out[4 * cj + 2]), "r"(out[4 * cj + 3]) : "memory");
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full0 + 8 * s);
-        }
+            };
+            ConvTable<BITS> T;
+            int cur_B = -1, next_B = -1;
+            __half sv_next = __float2half(0.f);
+            uint32_t zz_next = 0u;
 
-        // ---- epilogue: tensor memory -> fp16 -> global ----------------------------------------
-        if (ok && !mbar_wait(accum_bar, 0u)) ok = false;
-        if (ok) {
+            for (int kb = 2 * grp; kb < num_kb; kb = next_kb(kb)) {
+                const uint32_t it = it0 + (uint32_t)kb;
+                const int s = (int)(it % NSTAGE);
+                const uint32_t ph = (it / NSTAGE) & 1u;
+                if (valid) {
+                    const int Bk = block_of(kb);
+                    if (Bk != cur_B) {
+                        if (next_B != Bk) fetch_sz(Bk, sv_next, zz_next);
+                        cur_B = Bk;
+                        T.build(sv_next, zz_next);
+                    }
+                    // scale and zero-point of the block after this one are fetched one k-block ahead
+                    const int kn = next_kb(kb);
+                    const int Bn = block_of(kn);
+                    if (kn < num_kb && Bn != cur_B && Bn != next_B) {
+                        next_B = Bn;
+                        fetch_sz(Bn, sv_next, zz_next);
+                    }
+                }
+                if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
+                if (valid) {
+                    uint32_t w[BITS];
+                    const uint32_t pp = p_base + (uint32_t)s * P_STAGE_BYTES;
+#pragma unroll
+                    for (int i = 0; i < BITS; ++i)
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[i]) : "r"(pp + i * P_PLANE_BYTES) : "memory");
+                    uint32_t out[16];
+                    dequant_word<BITS>(w, T, out);
+                    const uint32_t row = b_base + (uint32_t)s * B_STAGE_BYTES;
+#pragma unroll
+                    for (int cj = 0; cj < 4; ++cj) {
+                        const uint32_t chunk = ((uint32_t)(4 * v + cj)) ^ xr;
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(row + chunk * 16u), "r"(out[4 * cj]),
+                                     "r"(out[4 * cj + 1]), "r"(out[4 * cj + 2]), "r"(out[4 * cj + 3]) : "memory");
+                    }
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full0 + 8 * s);
+            }
+            it0 += (uint32_t)num_kb;
+        }
+    } else {
+        // ---- epilogue: tensor memory -> fp16 -> global, one warp per quarter of the lanes --------
+        const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
+        uint32_t ti = 0;
+        while (ok && walk.next(t)) {
+            const uint32_t buf = ti & 1u, aph = (ti >> 1) & 1u;
+            if (!mbar_wait(accf0 + 8 * buf, aph)) { ok = false; break; }
             tcgen05_fence_after();
-            const int quarter = warp & 3;                 // tensor-memory lanes this warp may read
-            const int part = (warp - 2) >> 2;             // 32 of the tile's 128 columns
 #pragma unroll 1
             for (int h = 0; h < MH; ++h) {
-                const int m = tile_m * (BM * MH) + h * BM + quarter * 32 + lane;
-                const int col = part * 32;
-                uint32_t r[32];
-                tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * BN + col), r);
-                tcgen05_wait_ld();
-                if (m < p.M) {
-                    __half *dst = p.y + (size_t)m * p.N + (size_t)tile_n * BN + col;
+                const int m = t.tile_m * (BM * MH) + h * BM + quarter * 32 + lane;
+#pragma unroll 1
+                for (int col = 0; col < t.bn; col += 32) {
+                    uint32_t r[32];
+                    tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * ACC_COLS + (uint32_t)(h * BN + col), r);
+                    tcgen05_wait_ld();
+                    if (m < p.M) {
+                        __half *dst = p.y + (size_t)m * p.N + (size_t)t.col0 + col;
 #pragma unroll
-                    for (int g8 = 0; g8 < 4; ++g8) {
-                        if (tile_n * BN + col + 8 * g8 < p.N) {
-                            uint32_t h[4];
+                        for (int g8 = 0; g8 < 4; ++g8) {
+                            if (col + 8 * g8 < t.bn && t.col0 + col + 8 * g8 < p.N) {
+                                uint32_t hv[4];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const __half2 t = __floats2half2_rn(__uint_as_float(r[8 * g8 + 2 * e]),
-                                                                    __uint_as_float(r[8 * g8 + 2 * e + 1]));
-                                h[e] = *reinterpret_cast<const uint32_t *>(&t);
+                                for (int e = 0; e < 4; ++e) {
+                                    const __half2 hh = __floats2half2_rn(__uint_as_float(r[8 * g8 + 2 * e]),
+                                                                         __uint_as_float(r[8 * g8 + 2 * e + 1]));
+                                    hv[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + 8 * g8) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
                             }
-                            *reinterpret_cast<uint4 *>(dst + 8 * g8) = make_uint4(h[0], h[1], h[2], h[3]);
                         }
                     }
                 }
             }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+            ++ti;
         }
     }
 
@@ -496,7 +563,10 @@ tman_status launch_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, co
     auto kern = mpgemm_kernel<BITS, MH>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(MH, BITS)) != cudaSuccess)
         return TMAN_ERR_CUDA;
-    kern<<<p.tiles_m * p.tiles_n, GEMM_THREADS, smem_bytes(MH, BITS), s>>>(tmap_x, tmap_w, p);
+    // one CTA per SM (fewer when there are fewer items than that): every CTA walks through its items
+    long long grid = p.sms;
+    if (grid > (long long)p.tiles_m * p.R) grid = (long long)p.tiles_m * p.R;
+    kern<<<(unsigned)grid, GEMM_THREADS, smem_bytes(MH, BITS), s>>>(tmap_x, tmap_w, p);
     return launch_status();
 }
 
@@ -553,6 +623,22 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
     p.tiles_m = (M + BM * mh - 1) / (BM * mh);
     p.tiles_n = (N + BN - 1) / BN;
+    p.sms = sm_count();
+    if (p.sms <= 0) return TMAN_ERR_CUDA;
+    // Column ranges per row tile: the count that minimises (waves of items over the SMs) x (cost of an
+    // item), an item costing its width in 16-column units plus a fixed part (pipeline fill, epilogue).
+    {
+        const int n16 = (N + 15) / 16;
+        double best = 1e300;
+        p.R = 1;
+        for (int R = 1; R <= n16 && R <= 4096; ++R) {
+            const long long items = (long long)p.tiles_m * R;
+            const long long waves = (items + p.sms - 1) / p.sms;
+            const double width = (double)((n16 + R - 1) / R);
+            const double cost = (double)waves * (width + 2.0);
+            if (cost < best - 1e-9) { best = cost; p.R = R; }
+        }
+    }
     if (bits == 2) return launch_bits<2>(tmap, tmap_w, p, mh, s);
     if (bits == 3) return launch_bits<3>(tmap, tmap_w, p, mh, s);
     return launch_bits<4>(tmap, tmap_w, p, mh, s);
