@@ -162,7 +162,8 @@ struct UnitRegs {
 // tables; entry rows hold all 64 slots (slot = word + 16 * index byte) and the second half-warp
 // visits the index bytes of a word in the order 1,0,3,2, so that the 32 lanes still address 32
 // different banks.
-template <int BITS, int MT, int S, int PRE, int HALF>
+// GROUPED = 0: one matrix, the matrix index is a compile-time zero.
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED>
 __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -190,13 +191,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     {
         uint32_t hdr[kGemvMaxGroup][8];
 #pragma unroll
-        for (int g = 0; g < kGemvMaxGroup; ++g)
+        for (int g = 0; g < (GROUPED ? kGemvMaxGroup : 1); ++g)
             if (g < p.count) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q) hdr[g][q] = __ldg(reinterpret_cast<const uint32_t *>(p.packed[g]) + q);
             }
 #pragma unroll
-        for (int g = 0; g < kGemvMaxGroup; ++g)
+        for (int g = 0; g < (GROUPED ? kGemvMaxGroup : 1); ++g)
             if (g < p.count)
                 hdr_ok = hdr_ok && (hdr[g][0] == 0x4E414D54u) && (hdr[g][1] == 0x30303242u) && (hdr[g][2] == kVersion) &&
                          (hdr[g][3] == (uint32_t)p.K) && (hdr[g][4] == (uint32_t)p.Ng[g]) &&
@@ -212,15 +213,17 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     auto load_unit = [&](UnitRegs<BITS, S> &r, int wu) {
         const int u = min(wu, p.units - 1);
         int g = 0;
+        if constexpr (GROUPED) {
 #pragma unroll
-        for (int t = 1; t < kGemvMaxGroup; ++t) g += (t < p.count && u >= p.unit0[t]) ? 1 : 0;
-        const int lu = u - p.unit0[g];
+            for (int t = 1; t < kGemvMaxGroup; ++t) g += (t < p.count && u >= p.unit0[t]) ? 1 : 0;
+        }
+        const int lu = GROUPED ? u - p.unit0[g] : u;
         const int nstrips = p.Ng[g] >> 2;
         const uint8_t *pw = reinterpret_cast<const uint8_t *>(p.planes[g] + lane_word);
         const uint2 *psc = p.scales[g] + B;
         const uint16_t *pz = p.zeros[g] + B;
         r.g = g;
-        r.col = p.col0[g] + (lu * SUBS + sub) * S * 4;
+        r.col = (GROUPED ? p.col0[g] : 0) + (lu * SUBS + sub) * S * 4;
 #pragma unroll
         for (int s = 0; s < S; ++s) {
             const uint32_t nb = (uint32_t)min((lu * SUBS + sub) * S + s, nstrips - 1);
@@ -431,12 +434,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         LaneReduce<V1, PRE ? 2 : 1, W>::run(vals, v, base);
         const bool writer = (V >= W) ? true : (v < V);
         if (writer && wu < p.units) {
-            const int lim = p.col0[r.g] + p.Ng[r.g];   // end of this matrix's columns
+            const int g = GROUPED ? r.g : 0;
+            const int lim = GROUPED ? p.col0[g] + p.Ng[g] : p.N;   // end of this matrix's columns
 #pragma unroll
             for (int e = 0; e < NKEEP; ++e) {
                 const int idx = base + e, m = idx % MT, n = r.col + idx / MT;
                 if (n < lim && m < p.M) {
-                    if (p.nkappa == 1) p.y[r.g][(size_t)m * p.Ng[r.g] + (n - p.col0[r.g])] = __float2half_rn(vals[e]);
+                    if (p.nkappa == 1) p.y[g][(size_t)m * p.Ng[g] + (n - (GROUPED ? p.col0[g] : 0))] = __float2half_rn(vals[e]);
                     else p.partials[((size_t)kappa * MT + m) * p.N + n] = vals[e];
                 }
             }
@@ -506,8 +510,10 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 o.x = *reinterpret_cast<const uint32_t *>(&h01);
                 o.y = *reinterpret_cast<const uint32_t *>(&h23);
                 int g = 0;
+                if constexpr (GROUPED) {
 #pragma unroll
-                for (int t = 1; t < kGemvMaxGroup; ++t) g += (t < p.count && n >= p.col0[t]) ? 1 : 0;
+                    for (int t = 1; t < kGemvMaxGroup; ++t) g += (t < p.count && n >= p.col0[t]) ? 1 : 0;
+                }
                 *reinterpret_cast<uint2 *>(p.y[g] + (size_t)m * p.Ng[g] + (n - p.col0[g])) = o;
             }
         }
@@ -515,7 +521,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     }
 }
 
-template <int BITS, int MT, int S, int PRE, int HALF>
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED>
 static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
 {
     constexpr int W = HALF ? 16 : 32 / MT;
@@ -539,7 +545,7 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
         cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev) != cudaSuccess)
         return TMAN_ERR_CUDA;
     if ((uint32_t)reserved != kGemvSmemBase) return TMAN_ERR_UNSUPPORTED;
-    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF>;
+    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
         return TMAN_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -561,7 +567,8 @@ template <int BITS, int MT, int PRE>
 static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
 {
     constexpr int S = (MT == 1) ? ((BITS == 2) ? 2 : 1) : 1;
-    return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0>(p, sms, s);
+    if (p.count > 1) return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 1>(p, sms, s);
+    return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 0>(p, sms, s);
 }
 
 template <int BITS>
