@@ -27,20 +27,29 @@
 namespace tman {
 namespace {
 
-// A CTA multiplies MH row blocks of 128 tokens by one dequantized 128-column weight tile: every
+// A CTA multiplies MH row blocks of 128 tokens by one dequantized weight tile of up to BN columns: every
 // weight is rebuilt once per 128*MH tokens (MH = 2 halves the dequantization work per flop).
-constexpr int BM = 128, BN = 128, BK = 64;
-constexpr int NSTAGE = 4;
+// Two tile configurations.  WIDE: BN = 256, one MMA covers 256 output channels, so an activation tile
+// is read from shared memory once per 256 channels (shared-memory bandwidth is what bounds this
+// kernel); three stages of 72 KB fit and tensor memory holds one accumulator set.  Narrow: BN = 128,
+// four stages and two accumulator sets (the epilogue of a sub-tile overlaps the next one); used when
+// the output is so small that an SM's share is at most 128 columns wide.
+constexpr int BM = 128, BK = 64;
+template <int WIDE> struct Cfg {
+    static constexpr int BN = WIDE ? 256 : 128;
+    static constexpr int NSTAGE = WIDE ? 3 : 4;
+    static constexpr int NACC = WIDE ? 1 : 2;       // accumulator sets in tensor memory (MH * BN columns each)
+    static constexpr int B_STAGE_BYTES = BN * BK * 2;
+    static constexpr int P_PLANE_BYTES = (BN / 4) * (BK / 32) * 16;   // one plane of a packed tile
+};
 constexpr int A_HALF_BYTES = BM * BK * 2;
-constexpr int B_STAGE_BYTES = BN * BK * 2;
-constexpr int NUM_DEQ_WARPS = 8;                // warps that fill one weight tile
-constexpr int NUM_DEQ_GROUPS = 2;               // groups of such warps; they take turns, two k-blocks each
+constexpr int NUM_DEQ_WARPS = 16;               // each fills 16 columns of a weight tile
 constexpr int NUM_EPI_WARPS = 4;                // one per quarter of the tensor-memory lanes
-constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS * NUM_DEQ_GROUPS + NUM_EPI_WARPS);
-constexpr int P_PLANE_BYTES = (BN / 4) * (BK / 32) * 16;       // one plane of a packed tile: 32 strips x 2 words x 16 B
-constexpr int smem_bytes(int mh, int bits)
+constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS + NUM_EPI_WARPS);
+template <int WIDE> constexpr int smem_bytes(int mh, int bits)
 {
-    return NSTAGE * (mh * A_HALF_BYTES + B_STAGE_BYTES + bits * P_PLANE_BYTES) + 1024 /*align*/ + 256 /*barriers*/;
+    return Cfg<WIDE>::NSTAGE * (mh * A_HALF_BYTES + Cfg<WIDE>::B_STAGE_BYTES + bits * Cfg<WIDE>::P_PLANE_BYTES) +
+           1024 /*align*/ + 256 /*barriers*/;
 }
 
 struct GemmParams {
@@ -51,9 +60,10 @@ struct GemmParams {
     __half         *y;
     uint32_t       *status;
     int M, K, N, bits, group;
-    int tiles_m, tiles_n;
+    int tiles_m;
     int sms;
     int R;          // column ranges per row tile
+    int wide;       // tile configuration
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -281,16 +291,17 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
 
 // Work of a CTA.  The output is cut into row tiles of 128*MH tokens and, inside a row tile, into R
 // column ranges of (almost) equal width, a multiple of 16 columns.  The tiles_m * R items are dealt
-// to the CTAs round-robin; a CTA walks through an item in sub-tiles of at most 128 columns, again of
+// to the CTAs round-robin; a CTA walks through an item in sub-tiles of at most BN columns, again of
 // (almost) equal width.  Every role derives the same list from (blockIdx, gridDim).
 struct SubTile { int tile_m, col0, bn; };
 
 struct TileWalk {
-    int item, nitems, stride, tiles_m, R, n16;
+    int item, nitems, stride, tiles_m, R, n16, max16;
     int tm, lo, len, nsub, j;
-    __device__ TileWalk(const GemmParams &p, int cta, int ncta)
+    __device__ TileWalk(const GemmParams &p, int cta, int ncta, int bn_max)
         : item(cta - ncta), nitems(p.tiles_m * p.R), stride(ncta), tiles_m(p.tiles_m), R(p.R),
           n16((p.N + 15) >> 4),   // a last unit may reach 8 columns past N: computed, never stored
+          max16(bn_max / 16),
           tm(0), lo(0), len(0), nsub(0), j(0) {}
     __device__ bool next(SubTile &t)
     {
@@ -301,7 +312,7 @@ struct TileWalk {
             const int r = item / tiles_m;
             lo = (int)(((long long)n16 * r) / R);
             len = (int)(((long long)n16 * (r + 1)) / R) - lo;
-            nsub = (len + BN / 16 - 1) / (BN / 16);
+            nsub = (len + max16 - 1) / max16;
             j = 0;
         }
         const int u0 = lo + (len * j) / nsub, u1 = lo + (len * (j + 1)) / nsub;
@@ -313,13 +324,15 @@ struct TileWalk {
     }
 };
 
-template <int BITS, int MH>
+template <int BITS, int MH, int WIDE>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const GemmParams p)
 {
+    constexpr int BN = Cfg<WIDE>::BN, NSTAGE = Cfg<WIDE>::NSTAGE, NACC = Cfg<WIDE>::NACC;
+    constexpr int B_STAGE_BYTES = Cfg<WIDE>::B_STAGE_BYTES, P_PLANE_BYTES = Cfg<WIDE>::P_PLANE_BYTES;
     constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
     constexpr int ACC_COLS = MH * BN;                  // one fp32 accumulator of BN columns per row block
-    constexpr int TMEM_COLS = 2 * ACC_COLS;            // two sets: the epilogue of a sub-tile overlaps the next one
+    constexpr int TMEM_COLS = NACC * ACC_COLS;
     constexpr int P_STAGE_BYTES = BITS * P_PLANE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {
@@ -347,7 +360,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             mbar_init(full0 + 8 * s, NUM_DEQ_WARPS);
             mbar_init(empty0 + 8 * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < NACC; ++b) {
             mbar_init(accf0 + 8 * b, 1);
             mbar_init(acce0 + 8 * b, NUM_EPI_WARPS);
         }
@@ -363,7 +376,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
 
     bool ok = true;
-    TileWalk walk(p, (int)blockIdx.x, (int)gridDim.x);
+    TileWalk walk(p, (int)blockIdx.x, (int)gridDim.x, BN);
     SubTile t;
     if (warp == 0) {
         // ---- stage 1: activation tiles and packed weight tiles by TMA -------------------------
@@ -388,7 +401,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (lane == 0) {
             uint32_t it = 0, ti = 0;
             while (ok && walk.next(t)) {
-                const uint32_t buf = ti & 1u, aph = (ti >> 1) & 1u;
+                const uint32_t buf = ti % NACC, aph = (ti / NACC) & 1u;
                 if (!mbar_wait(acce0 + 8 * buf, aph ^ 1u)) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t idesc = (1u << 4) | ((uint32_t)(t.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -412,26 +425,32 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 ++ti;
             }
         }
-    } else if (warp < 2 + NUM_DEQ_WARPS * NUM_DEQ_GROUPS) {
+    } else if (warp < 2 + NUM_DEQ_WARPS) {
         // ---- stage 2: two-level lookup dequantization ----------------------------------------
         // A warp owns 16 columns and both plane words of a k-block: lane = (strip of the warp, word,
         // column of the strip).  With this split the 32 lanes read 32 different banks of the staged
         // plane words and write eight different 16-byte bank groups per quarter-warp.
-        const int wd = (warp - 2) & (NUM_DEQ_WARPS - 1), grp = (warp - 2) / NUM_DEQ_WARPS;
+        // Sub-tiles of at most 128 columns need only half of the warps per k-block: the two halves
+        // then take turns, two k-blocks each, so that all sixteen warps still share the work.
+        const int wd16 = warp - 2;
         const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
-        const int n_local = wd * 16 + sl * 4 + c;
         const int nblk = p.K / p.group;
         const int gshift = (p.group == 32) ? 5 : (p.group == 64) ? 6 : 7;
-        const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
-        const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
-        const uint32_t xr = (uint32_t)(n_local & 7);
-        const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
         auto block_of = [&](int kb) { return ((2 * kb + v) * 32) >> gshift; };
-        // k-blocks of this group: 2*grp, 2*grp+1, 2*grp+2*NUM_DEQ_GROUPS, ... (num_kb is even)
-        auto next_kb = [&](int kb) { return (kb & 1) ? kb + 2 * NUM_DEQ_GROUPS - 1 : kb + 1; };
 
         uint32_t it0 = 0;                                  // pipeline position of the sub-tile's first k-block
         while (ok && walk.next(t)) {
+            const int ngroups = (t.bn <= 128) ? 2 : 1;   // eight warps cover 128 columns
+            const int wd = (ngroups == 2) ? (wd16 & (NUM_DEQ_WARPS / 2 - 1)) : wd16;
+            const int grp = (ngroups == 2) ? wd16 / (NUM_DEQ_WARPS / 2) : 0;
+            const int n_local = wd * 16 + sl * 4 + c;
+            const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
+            const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
+            const uint32_t xr = (uint32_t)(n_local & 7);
+            const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
+            // k-blocks this warp works on: all of them, or every other pair (num_kb is even)
+            auto mine = [&](int kb) { return ngroups == 1 || ((kb >> 1) & 1) == grp; };
+            auto next_mine = [&](int kb) { return (ngroups == 1 || !(kb & 1)) ? kb + 1 : kb + 3; };
             const int n = t.col0 + n_local;
             const bool valid = n_local < t.bn && n < p.N;   // columns past the sub-tile are not used by the MMA
             const int nb = n >> 2;
@@ -450,11 +469,12 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             __half sv_next = __float2half(0.f);
             uint32_t zz_next = 0u;
 
-            for (int kb = 2 * grp; kb < num_kb; kb = next_kb(kb)) {
+            for (int kb = 0; kb < num_kb; ++kb) {
                 const uint32_t it = it0 + (uint32_t)kb;
                 const int s = (int)(it % NSTAGE);
                 const uint32_t ph = (it / NSTAGE) & 1u;
-                if (valid) {
+                const bool work = valid && mine(kb);
+                if (work) {
                     const int Bk = block_of(kb);
                     if (Bk != cur_B) {
                         if (next_B != Bk) fetch_sz(Bk, sv_next, zz_next);
@@ -462,7 +482,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         T.build(sv_next, zz_next);
                     }
                     // scale and zero-point of the block after this one are fetched one k-block ahead
-                    const int kn = next_kb(kb);
+                    const int kn = next_mine(kb);
                     const int Bn = block_of(kn);
                     if (kn < num_kb && Bn != cur_B && Bn != next_B) {
                         next_B = Bn;
@@ -470,7 +490,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     }
                 }
                 if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
-                if (valid) {
+                if (work) {
                     uint32_t w[BITS];
                     const uint32_t pp = p_base + (uint32_t)s * P_STAGE_BYTES;
 #pragma unroll
@@ -497,7 +517,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
         uint32_t ti = 0;
         while (ok && walk.next(t)) {
-            const uint32_t buf = ti & 1u, aph = (ti >> 1) & 1u;
+            const uint32_t buf = ti % NACC, aph = (ti / NACC) & 1u;
             if (!mbar_wait(accf0 + 8 * buf, aph)) { ok = false; break; }
             tcgen05_fence_after();
 #pragma unroll 1
@@ -557,23 +577,24 @@ EncodeTiledFn encode_fn()
     return reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-template <int BITS, int MH>
+template <int BITS, int MH, int WIDE>
 tman_status launch_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, cudaStream_t s)
 {
-    auto kern = mpgemm_kernel<BITS, MH>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(MH, BITS)) != cudaSuccess)
+    auto kern = mpgemm_kernel<BITS, MH, WIDE>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<WIDE>(MH, BITS)) != cudaSuccess)
         return TMAN_ERR_CUDA;
     // one CTA per SM (fewer when there are fewer items than that): every CTA walks through its items
     long long grid = p.sms;
     if (grid > (long long)p.tiles_m * p.R) grid = (long long)p.tiles_m * p.R;
-    kern<<<(unsigned)grid, GEMM_THREADS, smem_bytes(MH, BITS), s>>>(tmap_x, tmap_w, p);
+    kern<<<(unsigned)grid, GEMM_THREADS, smem_bytes<WIDE>(MH, BITS), s>>>(tmap_x, tmap_w, p);
     return launch_status();
 }
 
 template <int BITS>
 tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, int mh, cudaStream_t s)
 {
-    return mh == 2 ? launch_tile<BITS, 2>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1>(tmap_x, tmap_w, p, s);
+    if (p.wide) return mh == 2 ? launch_tile<BITS, 2, 1>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 1>(tmap_x, tmap_w, p, s);
+    return mh == 2 ? launch_tile<BITS, 2, 0>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 0>(tmap_x, tmap_w, p, s);
 }
 
 }  // namespace
@@ -599,20 +620,6 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
 
     Layout L = make_layout(K, N, bits, group);
     const uint8_t *pk = static_cast<const uint8_t *>(packed);
-    // the bit-plane words as a 3-D array of 32-bit elements: (word and column inside a strip's plane
-    // row, plane, strip); one box = the two words of a k-block for 32 strips of one plane
-    CUtensorMap tmap_w;
-    {
-        const cuuint64_t wt = (cuuint64_t)(K / 32);
-        const cuuint64_t wdims[3] = {wt * 4, (cuuint64_t)bits, (cuuint64_t)(N / 4)};
-        const cuuint64_t wstrides[2] = {wt * 16, wt * 16 * (cuuint64_t)bits};
-        const cuuint32_t wbox[3] = {(cuuint32_t)(BK / 8), 1, (cuuint32_t)(BN / 4)};
-        const cuuint32_t westr[3] = {1, 1, 1};
-        if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t *>(pk + L.planes_off), wdims, wstrides,
-                wbox, westr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return TMAN_ERR_CUDA;
-    }
     GemmParams p;
     p.packed = pk;
     p.planes = reinterpret_cast<const uint32_t *>(pk + L.planes_off);
@@ -622,22 +629,42 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.status = static_cast<uint32_t *>(ws);
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
     p.tiles_m = (M + BM * mh - 1) / (BM * mh);
-    p.tiles_n = (N + BN - 1) / BN;
     p.sms = sm_count();
     if (p.sms <= 0) return TMAN_ERR_CUDA;
-    // Column ranges per row tile: the count that minimises (waves of items over the SMs) x (cost of an
-    // item), an item costing its width in 16-column units plus a fixed part (pipeline fill, epilogue).
+    // Tile configuration and column ranges per row tile: the pair that minimises (waves of items over
+    // the SMs) x (cost of an item).  A sub-tile of w 16-column units costs about w + 10 units of
+    // shared-memory traffic per k-block (the activation tile is written once and read once per MMA
+    // whatever the width), and a wide sub-tile holds twice as many units as a narrow one.
     {
         const int n16 = (N + 15) / 16;
         double best = 1e300;
         p.R = 1;
-        for (int R = 1; R <= n16 && R <= 4096; ++R) {
-            const long long items = (long long)p.tiles_m * R;
-            const long long waves = (items + p.sms - 1) / p.sms;
-            const double width = (double)((n16 + R - 1) / R);
-            const double cost = (double)waves * (width + 2.0);
-            if (cost < best - 1e-9) { best = cost; p.R = R; }
+        p.wide = 0;
+        for (int wide = 0; wide < 2; ++wide) {
+            const int maxw = (wide ? Cfg<1>::BN : Cfg<0>::BN) / 16;
+            for (int R = 1; R <= n16 && R <= 4096; ++R) {
+                const long long items = (long long)p.tiles_m * R;
+                const long long waves = (items + p.sms - 1) / p.sms;
+                const int w16 = (n16 + R - 1) / R;
+                const int nsub = (w16 + maxw - 1) / maxw;
+                const double cost = (double)waves * (w16 + 10.0 * nsub);
+                if (cost < best - 1e-9) { best = cost; p.R = R; p.wide = wide; }
+            }
         }
+    }
+    // the bit-plane words as a 3-D array of 32-bit elements: (word and column inside a strip's plane
+    // row, plane, strip); one box = the two words of a k-block for the strips of a tile, one plane
+    CUtensorMap tmap_w;
+    {
+        const cuuint64_t wt = (cuuint64_t)(K / 32);
+        const cuuint64_t wdims[3] = {wt * 4, (cuuint64_t)bits, (cuuint64_t)(N / 4)};
+        const cuuint64_t wstrides[2] = {wt * 16, wt * 16 * (cuuint64_t)bits};
+        const cuuint32_t wbox[3] = {(cuuint32_t)(BK / 8), 1, (cuuint32_t)((p.wide ? Cfg<1>::BN : Cfg<0>::BN) / 4)};
+        const cuuint32_t westr[3] = {1, 1, 1};
+        if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t *>(pk + L.planes_off), wdims, wstrides,
+                wbox, westr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TMAN_ERR_CUDA;
     }
     if (bits == 2) return launch_bits<2>(tmap, tmap_w, p, mh, s);
     if (bits == 3) return launch_bits<3>(tmap, tmap_w, p, mh, s);
