@@ -16,7 +16,7 @@
 //                        tensor core reads;
 //   * warp 1, one lane : tcgen05.mma (M128 N<=128 K16, fp16 x fp16 -> fp32 in tensor memory), one
 //                        per row block; tcgen05.commit hands the stage back;
-//   * warps 18..21     : epilogue of the previous tile (tcgen05.ld, round to fp16, store) while the
+//   * warps 18..25     : epilogue of the previous tile (tcgen05.ld, round to fp16, store) while the
 //                        next tile accumulates into the second set of tensor-memory columns.
 // Every wait is bounded: when a bound is hit the kernel records TMAN_ERR_TIMEOUT, stops issuing
 // work, and still reaches the common tear-down that frees tensor memory.
@@ -44,7 +44,7 @@ template <int WIDE> struct Cfg {
 };
 constexpr int A_HALF_BYTES = BM * BK * 2;
 constexpr int NUM_DEQ_WARPS = 16;               // each fills 16 columns of a weight tile
-constexpr int NUM_EPI_WARPS = 4;                // one per quarter of the tensor-memory lanes
+constexpr int NUM_EPI_WARPS = 8;                // two per quarter of the tensor-memory lanes (alternate 32-column chunks)
 constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS + NUM_EPI_WARPS);
 template <int WIDE> constexpr int smem_bytes(int mh, int bits)
 {
@@ -515,6 +515,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     } else {
         // ---- epilogue: tensor memory -> fp16 -> global, one warp per quarter of the lanes --------
         const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
+        const int epart = (warp - 2 - NUM_DEQ_WARPS) >> 2; // which of the quarter's warps
         uint32_t ti = 0;
         while (ok && walk.next(t)) {
             const uint32_t buf = ti % NACC, aph = (ti / NACC) & 1u;
@@ -524,7 +525,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             for (int h = 0; h < MH; ++h) {
                 const int m = t.tile_m * (BM * MH) + h * BM + quarter * 32 + lane;
 #pragma unroll 1
-                for (int col = 0; col < t.bn; col += 32) {
+                for (int col = 32 * epart; col < t.bn; col += 32 * (NUM_EPI_WARPS / 4)) {
                     uint32_t r[32];
                     tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * ACC_COLS + (uint32_t)(h * BN + col), r);
                     tcgen05_wait_ld();
