@@ -22,8 +22,10 @@
 // "ready" flag, so no fence and no counter sits between the last lookup and the output; the poll
 // is bounded and reports TMAN_ERR_TIMEOUT.
 //
-// Streaming.  A warp works through small units (a few strips of four columns) and keeps the next
-// unit's plane words in a second set of registers, so that HBM reads overlap the lookups.  The
+// Streaming.  A warp works through units (a few strips of four columns).  With one activation row
+// every strip's registers are refilled with the next unit's strip as soon as its lookups are done;
+// with more rows the next unit sits in a second set of registers.  Either way HBM reads overlap the
+// lookups.  The
 // first loads are issued before the kernel waits for the previous kernel in the stream
 // (programmatic dependent launch): weights are constant input and the host has checked that
 // every read derived from (K, N, bits, group) is in bounds.
@@ -163,7 +165,9 @@ struct UnitRegs {
 // visits the index bytes of a word in the order 1,0,3,2, so that the 32 lanes still address 32
 // different banks.
 // GROUPED = 0: one matrix, the matrix index is a compile-time zero.
-template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED>
+// ROLL: one set of unit registers; every strip's registers are refilled with the next unit's strip as
+// soon as its lookups are done (larger units, fewer per-unit fixed costs, same bytes in flight).
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL>
 __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -210,39 +214,46 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     const uint32_t lane_word = (uint32_t)(word0 + (active ? v : 0));
     const uint32_t row_bytes = (uint32_t)words_total * 16u;      // one plane of one strip
     const uint32_t strip_bytes = row_bytes * BITS;
-    auto load_unit = [&](UnitRegs<BITS, S> &r, int wu) {
+    struct UnitAddr { const uint8_t *pw; const uint2 *psc; const uint16_t *pz; int lu, nstrips; };
+    auto unit_addr = [&](UnitRegs<BITS, S> &r, int wu) {
         const int u = min(wu, p.units - 1);
         int g = 0;
         if constexpr (GROUPED) {
 #pragma unroll
             for (int t = 1; t < kGemvMaxGroup; ++t) g += (t < p.count && u >= p.unit0[t]) ? 1 : 0;
         }
-        const int lu = GROUPED ? u - p.unit0[g] : u;
-        const int nstrips = p.Ng[g] >> 2;
-        const uint8_t *pw = reinterpret_cast<const uint8_t *>(p.planes[g] + lane_word);
-        const uint2 *psc = p.scales[g] + B;
-        const uint16_t *pz = p.zeros[g] + B;
+        UnitAddr a;
+        a.lu = GROUPED ? u - p.unit0[g] : u;
+        a.nstrips = p.Ng[g] >> 2;
+        a.pw = reinterpret_cast<const uint8_t *>(p.planes[g] + lane_word);
+        a.psc = p.scales[g] + B;
+        a.pz = p.zeros[g] + B;
         r.g = g;
-        r.col = (GROUPED ? p.col0[g] : 0) + (lu * SUBS + sub) * S * 4;
+        r.col = (GROUPED ? p.col0[g] : 0) + (a.lu * SUBS + sub) * S * 4;
+        return a;
+    };
+    auto load_strip = [&](UnitRegs<BITS, S> &r, int s, const UnitAddr &a) {
+        const uint32_t nb = (uint32_t)min((a.lu * SUBS + sub) * S + s, a.nstrips - 1);
+        const uint8_t *q = a.pw + (size_t)nb * strip_bytes;
 #pragma unroll
-        for (int s = 0; s < S; ++s) {
-            const uint32_t nb = (uint32_t)min((lu * SUBS + sub) * S + s, nstrips - 1);
-            const uint8_t *q = pw + (size_t)nb * strip_bytes;
-#pragma unroll
-            for (int i = 0; i < BITS; ++i) {
-                r.w[s][i] = __ldcs(reinterpret_cast<const uint4 *>(q));
-                q += row_bytes;
-            }
-            r.sc[s] = __ldg(psc + (size_t)nb * (uint32_t)nblk);
-            r.z[s] = __ldg(pz + (size_t)nb * (uint32_t)nblk);
+        for (int i = 0; i < BITS; ++i) {
+            r.w[s][i] = __ldcs(reinterpret_cast<const uint4 *>(q));
+            q += row_bytes;
         }
+        r.sc[s] = __ldg(a.psc + (size_t)nb * (uint32_t)nblk);
+        r.z[s] = __ldg(a.pz + (size_t)nb * (uint32_t)nblk);
+    };
+    auto load_unit = [&](UnitRegs<BITS, S> &r, int wu) {
+        const UnitAddr a = unit_addr(r, wu);
+#pragma unroll
+        for (int s = 0; s < S; ++s) load_strip(r, s, a);
     };
 
     // Issue the first unit's weight loads before anything else: the packed buffer is constant
     // input and packed_bytes was checked on the host, so these reads are in bounds whatever the
     // header says.  Their latency overlaps the table build.
     const int wu0 = j + p.P * warp, wstride = p.P * kGemvWarps;
-    UnitRegs<BITS, S> regs[2];
+    UnitRegs<BITS, S> regs[ROLL ? 1 : 2];
     load_unit(regs[0], wu0);
 
     // Everything below may depend on the previous kernel in the stream (activations, workspace).
@@ -255,7 +266,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         const int gv = slot & 15, gc = slot >> 4;
         uint4 raw = make_uint4(0u, 0u, 0u, 0u);
         if (gv < nwords) raw = __ldg(reinterpret_cast<const uint4 *>(p.x + (size_t)(word0 + gv) * 32 + gc * 8));
-        load_unit(regs[1], wu0 + wstride);
+        if constexpr (!ROLL) load_unit(regs[1], wu0 + wstride);
         float xv[8];
         const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
 #pragma unroll
@@ -289,7 +300,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     #pragma unroll
             for (int c = 0; c < 4; ++c) xraw[c] = __ldg(px + c);
         }
-        load_unit(regs[1], wu0 + wstride);
+        if constexpr (!ROLL) load_unit(regs[1], wu0 + wstride);
 
         // ---- phase A: activation tables (paper Sec. 2.2; one table per 8 activations, 256 entries,
         // entry = 16-entry table of the low four + sum of the selected high four) -----------------
@@ -357,10 +368,18 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     }
 
     // ---- phase B: lookups, shift-accumulate, scale and zero-point (paper Sec. 4.3) --------------
-    auto compute_unit = [&](const UnitRegs<BITS, S> &r, int wu) {
+    auto compute_unit = [&](UnitRegs<BITS, S> &r, int wu, int next_wu) {
         float vals[V];
+        // what the end of the unit needs survives the refill of the strip registers
+        uint2 sc_s[S];
+        uint32_t z_s[S];
 #pragma unroll
-        for (int s = 0; s < S; ++s)
+        for (int s = 0; s < S; ++s) { sc_s[s] = r.sc[s]; z_s[s] = r.z[s]; }
+        const int g_u = r.g, col_u = r.col;
+        UnitAddr nxt;
+        if constexpr (ROLL) nxt = unit_addr(r, next_wu);
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
                 float a[MT];
@@ -389,6 +408,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
                 for (int m = 0; m < MT; ++m) vals[(s * 4 + c4) * MT + m] = a[m];
             }
+            if constexpr (ROLL) load_strip(r, s, nxt);
+        }
 
         // lanes v and v^1 hold the two words of one block: add them first, keeping half the columns
         int base = 0;
@@ -399,8 +420,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             constexpr int S1 = PRE ? S / 2 : S;
 #pragma unroll
             for (int s = 0; s < S1; ++s) {
-                const uint2 scq = up ? r.sc[s + (PRE ? S1 : 0)] : r.sc[s];
-                const uint32_t zq = up ? r.z[s + (PRE ? S1 : 0)] : r.z[s];
+                const uint2 scq = up ? sc_s[s + (PRE ? S1 : 0)] : sc_s[s];
+                const uint32_t zq = up ? z_s[s + (PRE ? S1 : 0)] : z_s[s];
                 const __half2 s01 = *reinterpret_cast<const __half2 *>(&scq.x);
                 const __half2 s23 = *reinterpret_cast<const __half2 *>(&scq.y);
                 const float sc[4] = {__low2float(s01), __high2float(s01), __low2float(s23), __high2float(s23)};
@@ -416,8 +437,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             }
         } else {
             // one strip, two of its four columns left
-            const uint32_t scq = up ? r.sc[0].y : r.sc[0].x;
-            const uint32_t zq = up ? (r.z[0] >> 8) : r.z[0];
+            const uint32_t scq = up ? sc_s[0].y : sc_s[0].x;
+            const uint32_t zq = up ? (z_s[0] >> 8) : z_s[0];
             const __half2 s01 = *reinterpret_cast<const __half2 *>(&scq);
             const float sc[2] = {__low2float(s01), __high2float(s01)};
 #pragma unroll
@@ -434,11 +455,11 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         LaneReduce<V1, PRE ? 2 : 1, W>::run(vals, v, base);
         const bool writer = (V >= W) ? true : (v < V);
         if (writer && wu < p.units) {
-            const int g = GROUPED ? r.g : 0;
+            const int g = GROUPED ? g_u : 0;
             const int lim = GROUPED ? p.col0[g] + p.Ng[g] : p.N;   // end of this matrix's columns
 #pragma unroll
             for (int e = 0; e < NKEEP; ++e) {
-                const int idx = base + e, m = idx % MT, n = r.col + idx / MT;
+                const int idx = base + e, m = idx % MT, n = col_u + idx / MT;
                 if (n < lim && m < p.M) {
                     if (p.nkappa == 1) p.y[g][(size_t)m * p.Ng[g] + (n - (GROUPED ? p.col0[g] : 0))] = __float2half_rn(vals[e]);
                     else p.partials[((size_t)kappa * MT + m) * p.N + n] = vals[e];
@@ -447,12 +468,16 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         }
     };
 
-    for (int wu = wu0; wu < p.units; wu += 2 * wstride) {
-        compute_unit(regs[0], wu);
-        load_unit(regs[0], wu + 2 * wstride);
-        if (wu + wstride >= p.units) break;            // uniform over the warp
-        compute_unit(regs[1], wu + wstride);
-        load_unit(regs[1], wu + 3 * wstride);
+    if constexpr (ROLL) {
+        for (int wu = wu0; wu < p.units; wu += wstride) compute_unit(regs[0], wu, wu + wstride);
+    } else {
+        for (int wu = wu0; wu < p.units; wu += 2 * wstride) {
+            compute_unit(regs[0], wu, 0);
+            load_unit(regs[0], wu + 2 * wstride);
+            if (wu + wstride >= p.units) break;        // uniform over the warp
+            compute_unit(regs[1], wu + wstride, 0);
+            load_unit(regs[1], wu + 3 * wstride);
+        }
     }
 
     // ---- combine K-slices: every CTA polls the partial sums of its share of the columns ----------
@@ -521,7 +546,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     }
 }
 
-template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED>
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL>
 static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
 {
     constexpr int W = HALF ? 16 : 32 / MT;
@@ -545,7 +570,7 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
         cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev) != cudaSuccess)
         return TMAN_ERR_CUDA;
     if ((uint32_t)reserved != kGemvSmemBase) return TMAN_ERR_UNSUPPORTED;
-    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED>;
+    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED, ROLL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
         return TMAN_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -562,13 +587,14 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     return TMAN_OK;
 }
 
-// strips per unit: small enough that two units fit in registers, large enough for V >= 4
 template <int BITS, int MT, int PRE>
 static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
 {
-    constexpr int S = (MT == 1) ? ((BITS == 2) ? 2 : 1) : 1;
-    if (p.count > 1) return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 1>(p, sms, s);
-    return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 0>(p, sms, s);
+    // one row: large units on one rolling set of registers; more rows: small double-buffered units
+    constexpr int ROLL = (MT == 1) ? 1 : 0;
+    constexpr int S = (MT == 1) ? ((BITS == 2) ? 4 : 2) : 1;
+    if (p.count > 1) return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 1, ROLL>(p, sms, s);
+    return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 0, ROLL>(p, sms, s);
 }
 
 template <int BITS>
