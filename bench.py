@@ -192,7 +192,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    from paper_2511_11248_b200 import binding as B, helpers as H, synth
+    from paper_2511_11248_b200 import binding as B, helpers as H, replicas, synth
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -265,13 +265,9 @@ def run_ours(args):
         ev1.record()
         torch.cuda.synchronize()
     barrier()
-    ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = replicas.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
     sec_step = ms / 1e3 / steps
-    value = world * wbytes_step / sec_step / 1e9
+    value = replicas.whole_job_rate(wbytes_step, sec_step, world) / 1e9
     st = [B.tman_read_status(e[5]) for s in sets for e in s]
     assert all(v == 0 for v in st), f"device status {st}"
 
@@ -299,12 +295,8 @@ def run_ours(args):
         e2e_step(i)
     ev1.record()
     torch.cuda.synchronize()
-    e2e_ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_val = world * wbytes_step / (e2e_ms / 1e3 / e2e_steps) / 1e9
+    e2e_ms = replicas.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
+    e2e_val = replicas.whole_job_rate(wbytes_step, e2e_ms / 1e3 / e2e_steps, world) / 1e9
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
