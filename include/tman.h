@@ -80,11 +80,13 @@ tman_status tman_read_status(const void *workspace, int *out_status /*host*/,
  * zeros  uint8 [K/group][N], values in [0, 2^bits)
  * packed: output, packed_bytes >= tman_packed_bytes(...), 256-byte aligned.
  * Layout written (little endian):
- *   header (256 B): "TMANB200", u32 version=1, u32 K, N, bits, group, lut_g=4,
+ *   header (256 B): "TMANB200", u32 version=2, u32 K, N, bits, group, lut_g=4,
  *                   u64 planes_off, scales_off, zeros_off, total_bytes
- *   planes: u32 word[((nb*bits + i)*(K/32) + v)*4 + c], n = 4*nb + c; bit r of the word is
- *           bit i of q[32*v + r][n].  Nibble e of the word is the paper's 4-bit table index
- *           of plane i for activations 32v+4e .. 32v+4e+3.
+ *   planes: u32 word[((nb*bits + i)*(K/32) + v)*4 + c], n = 4*nb + c; the word holds bit i of the 32
+ *           codes q[32*v .. 32*v+31][n], permuted: weight 32*v + 8*ph + j sits at bit 4*j + ph
+ *           (ph < 4, j < 8).  Byte e of the word is an 8-bit table index over the activations
+ *           32*v + 8*ph + 2*e + hi (index bit 4*hi + ph); its nibbles are 4-bit indices in the
+ *           paper's sense.  The permutation is what lets the prefill path rebuild codes in k order.
  *   scales: fp16 [((nb*(K/group) + B)*4 + c]
  *   zeros : u16  [nb*(K/group) + B], nibble c = z[B][4*nb + c]                              */
 tman_status tman_pack_weights(const uint8_t *codes, const void *scales_f16, const uint8_t *zeros,

@@ -224,6 +224,12 @@ size_t oracle_packed_bytes(int K, int N, int bits, int G)
     return ORACLE_HDR_BYTES + up256(planes) + up256(scales) + up256(zeros);
 }
 
+/* Bit position, inside a plane word, of the weight with k % 32 == r.  The 32 weights of a word are
+ * stored permuted (paper Sec. 4.1: weights are permuted offline so that the on-the-fly repacking of
+ * the prefill path is cheap): weight r = 8*ph + j sits at bit 4*j + ph, so that the four nibble-packed
+ * code words of the repacking step come out in consecutive-k order. */
+static int plane_bit(int r) { return 4 * (r & 7) + (r >> 3); }
+
 static void put32(uint8_t *p, uint32_t v) { memcpy(p, &v, 4); }
 static void put64(uint8_t *p, uint64_t v) { memcpy(p, &v, 8); }
 
@@ -239,7 +245,7 @@ void oracle_pack(const uint8_t *q, const uint16_t *s, const uint8_t *z,
     int nb, i, v, c, r, B;
     memset(out, 0, total);
     memcpy(out, "TMANB200", 8);
-    put32(out + 8, 1);
+    put32(out + 8, 2);
     put32(out + 12, (uint32_t)K);
     put32(out + 16, (uint32_t)N);
     put32(out + 20, (uint32_t)bits);
@@ -249,14 +255,14 @@ void oracle_pack(const uint8_t *q, const uint16_t *s, const uint8_t *z,
     put64(out + 40, scales_off);
     put64(out + 48, zeros_off);
     put64(out + 56, total);
-    /* plane words: bit r of word (strip nb, plane i, v, c) = bit i of q[32v + r][4nb + c] */
+    /* plane words: bit plane_bit(r) of word (strip nb, plane i, v, c) = bit i of q[32v + r][4nb + c] */
     for (nb = 0; nb < N / 4; ++nb)
         for (i = 0; i < bits; ++i)
             for (v = 0; v < K / 32; ++v)
                 for (c = 0; c < 4; ++c) {
                     uint32_t w = 0;
                     for (r = 0; r < 32; ++r)
-                        w |= (uint32_t)((q[(size_t)(32 * v + r) * N + 4 * nb + c] >> i) & 1) << r;
+                        w |= (uint32_t)((q[(size_t)(32 * v + r) * N + 4 * nb + c] >> i) & 1) << plane_bit(r);
                     put32(out + planes_off +
                           4 * ((((size_t)nb * bits + i) * (K / 32) + v) * 4 + c), w);
                 }
@@ -287,7 +293,7 @@ int oracle_unpack(const uint8_t *in, uint8_t *q, uint16_t *s, uint8_t *z)
     memcpy(&planes_off, in + 32, 8);
     memcpy(&scales_off, in + 40, 8);
     memcpy(&zeros_off, in + 48, 8);
-    if (ver != 1) return 2;
+    if (ver != 2) return 2;
     memset(q, 0, (size_t)K * N);
     for (nb = 0; nb < N / 4; ++nb)
         for (i = 0; i < bits; ++i)
@@ -298,7 +304,7 @@ int oracle_unpack(const uint8_t *in, uint8_t *q, uint16_t *s, uint8_t *z)
                            4 * ((((size_t)nb * bits + i) * (K / 32) + v) * 4 + c), 4);
                     for (r = 0; r < 32; ++r)
                         q[(size_t)(32 * v + r) * N + 4 * nb + c] |=
-                            (uint8_t)(((w >> r) & 1) << i);
+                            (uint8_t)(((w >> plane_bit((int)r)) & 1) << i);
                 }
     for (nb = 0; nb < N / 4; ++nb)
         for (B = 0; B < K / G; ++B) {

@@ -21,7 +21,11 @@ struct PackedHeader {
 static_assert(sizeof(PackedHeader) == 64, "header fields occupy the first 64 bytes");
 
 constexpr size_t   kHeaderBytes = 256;
-constexpr uint32_t kVersion = 1;
+constexpr uint32_t kVersion = 2;
+
+// Bit of a plane word that holds the weight with k % 32 == r: weight 8*ph + j sits at bit 4*j + ph
+// (an offline permutation, paper Sec. 4.1, that makes the prefill repacking come out in k order).
+__host__ __device__ constexpr int plane_bit(int r) { return 4 * (r & 7) + (r >> 3); }
 
 __host__ __device__ inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 

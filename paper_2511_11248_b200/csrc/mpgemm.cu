@@ -241,13 +241,14 @@ struct ConvTable {
     }
 };
 
-// 32 weights of one column (one plane word per bit) -> 16 half2 in natural k order.
+// 32 weights of one column (one plane word per bit) -> 16 half2 in k order.
 template <int BITS>
 __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const ConvTable<BITS> &T, uint32_t (&out)[16])
 {
-    // level 1 (bit repacking): X[ph] nibble j = code of weight 4j + ph.  A 4 x 4 bit-block
-    // transpose of the plane words: first planes 0/1 and 2/3 are interleaved bit by bit, then the
-    // two results two bits by two bits (each step is one shift and one bit-select).
+    // level 1 (bit repacking): X[ph] nibble j = code of the weight at word bit 4j + ph, which the
+    // packed format makes weight 8*ph + j: X[ph] holds weights 8ph .. 8ph+7 in order.  A 4 x 4
+    // bit-block transpose of the plane words: first planes 0/1 and 2/3 are interleaved bit by bit,
+    // then the two results two bits by two bits (each step is one shift and one bit-select).
     auto bsel = [](uint32_t m, uint32_t a, uint32_t b) { return (a & m) | (b & ~m); };
     uint32_t X[4];
     {
@@ -267,25 +268,16 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
             X[3] = (a1 >> 2) & 0x33333333u;
         }
     }
-    // level 2 (conversion table) and re-pairing into adjacent k
-    uint32_t A[4][2], Bv[4][2];
+    // level 2 (conversion table): four codes per lookup, then low and high bytes are interleaved
+    // into two half2 of adjacent weights
 #pragma unroll
     for (int ph = 0; ph < 4; ++ph)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             uint32_t lb, hb;
             T.lookup(X[ph] >> (16 * h), lb, hb);
-            A[ph][h] = __byte_perm(lb, hb, 0x5140);    // weights k0, k0+4   (k0 = 16h + ph)
-            Bv[ph][h] = __byte_perm(lb, hb, 0x7362);   // weights k0+8, k0+12
-        }
-#pragma unroll
-    for (int h = 0; h < 2; ++h)
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            out[8 * h + q]     = __byte_perm(A[2 * q][h], A[2 * q + 1][h], 0x5410);
-            out[8 * h + 2 + q] = __byte_perm(A[2 * q][h], A[2 * q + 1][h], 0x7632);
-            out[8 * h + 4 + q] = __byte_perm(Bv[2 * q][h], Bv[2 * q + 1][h], 0x5410);
-            out[8 * h + 6 + q] = __byte_perm(Bv[2 * q][h], Bv[2 * q + 1][h], 0x7632);
+            out[4 * ph + 2 * h]     = __byte_perm(lb, hb, 0x5140);    // weights k0, k0+1   (k0 = 8ph + 4h)
+            out[4 * ph + 2 * h + 1] = __byte_perm(lb, hb, 0x7362);    // weights k0+2, k0+3
         }
 }
 

@@ -264,16 +264,21 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         // three high index bits of its 32 entries
         const int slot = tid & 63, chunk = tid >> 6;
         const int gv = slot & 15, gc = slot >> 4;
-        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-        if (gv < nwords) raw = __ldg(reinterpret_cast<const uint4 *>(p.x + (size_t)(word0 + gv) * 32 + gc * 8));
+        // index bit q of byte gc is word bit 8*gc + q, i.e. the weight 8*(q & 3) + 2*gc + (q >> 2)
+        __half2 raw[4];
+#pragma unroll
+        for (int ph = 0; ph < 4; ++ph) {
+            raw[ph] = __floats2half2_rn(0.f, 0.f);
+            if (gv < nwords)
+                raw[ph] = __ldg(reinterpret_cast<const __half2 *>(p.x + (size_t)(word0 + gv) * 32 + 8 * ph + 2 * gc));
+        }
         if constexpr (!ROLL) load_unit(regs[1], wu0 + wstride);
         float xv[8];
-        const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float2 f = __half22float2(h2[q]);
-            xv[2 * q] = f.x;
-            xv[2 * q + 1] = f.y;
+        for (int ph = 0; ph < 4; ++ph) {
+            const float2 f = __half22float2(raw[ph]);
+            xv[ph] = f.x;
+            xv[ph + 4] = f.y;
         }
         float lo[16];
         lut16(xv[0], xv[1], xv[2], xv[3], lo);
@@ -293,11 +298,11 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         const int vb = lane / MT, mb = lane % MT;
         const bool live = (vb < nwords) && (mb < p.M);
         uint4 xraw[4];
-    #pragma unroll
+#pragma unroll
         for (int c = 0; c < 4; ++c) xraw[c] = make_uint4(0u, 0u, 0u, 0u);
         if (live) {
             const uint4 *px = reinterpret_cast<const uint4 *>(p.x + (size_t)mb * p.K + (size_t)(word0 + vb) * 32);
-    #pragma unroll
+#pragma unroll
             for (int c = 0; c < 4; ++c) xraw[c] = __ldg(px + c);
         }
         if constexpr (!ROLL) load_unit(regs[1], wu0 + wstride);
@@ -307,15 +312,16 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         {
             // warp w fills the entries whose high index nibble is w, for all four groups of the word
             const int ph = warp;
-    #pragma unroll
+#pragma unroll
             for (int c = 0; c < 4; ++c) {
+                // index bit q of byte c is word bit 8*c + q, i.e. the weight 8*(q & 3) + 2*c + (q >> 2):
+                // the c-th pair of each quarter of the word
                 float xv[8];
-                const __half2 *h2 = reinterpret_cast<const __half2 *>(&xraw[c]);
-    #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const float2 f = __half22float2(h2[q]);
-                    xv[2 * q] = f.x;
-                    xv[2 * q + 1] = f.y;
+#pragma unroll
+                for (int ph = 0; ph < 4; ++ph) {
+                    const float2 f = __half22float2(reinterpret_cast<const __half2 *>(&xraw[ph])[c]);
+                    xv[ph] = f.x;
+                    xv[ph + 4] = f.y;
                 }
                 float lo[16];
                 lut16(xv[0], xv[1], xv[2], xv[3], lo);
@@ -325,7 +331,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 if (ph & 4) hi += xv[6];
                 if (ph & 8) hi += xv[7];
                 uint8_t *dst = smem + table_imm(c) + (uint32_t)(ph * 16) * 256u + (uint32_t)lane * 4u;
-    #pragma unroll
+#pragma unroll
                 for (int pl = 0; pl < 16; ++pl)
                     *reinterpret_cast<float *>(dst + pl * 256) = lo[pl] + hi;
             }

@@ -18,7 +18,7 @@ __global__ void pack_planes_kernel(const uint8_t *__restrict__ codes, uint32_t *
     for (int r = 0; r < 32; ++r) {
         uint32_t q = codes[(size_t)(32 * v + r) * N + n];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) w[i] |= ((q >> i) & 1u) << r;
+        for (int i = 0; i < 4; ++i) w[i] |= ((q >> i) & 1u) << plane_bit(r);
     }
     int nb = n >> 2, c = n & 3;
     for (int i = 0; i < bits; ++i)
@@ -117,7 +117,7 @@ __global__ void unpack_kernel(const uint8_t *__restrict__ packed, uint8_t *__res
         for (int r = 0; r < 32; ++r) {
             uint32_t q = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) q |= ((w[i] >> r) & 1u) << i;
+            for (int i = 0; i < 4; ++i) q |= ((w[i] >> plane_bit(r)) & 1u) << i;
             codes[(size_t)(32 * v + r) * N + n] = (uint8_t)q;
         }
     }
@@ -143,7 +143,8 @@ tman_status launch_unpack(const void *packed, int K, int N, int bits, int group,
 }
 
 // ---- test-only extractors ------------------------------------------------------------------
-// idx[i][t][n] = nibble (t % 8) of plane word (i, t / 8, n): what the kernels use as table index.
+// idx[i][t][n] = the 4-bit table index of activations 4t .. 4t+3 (plane i, column n), gathered from
+// the bits of plane word (i, t / 8, n) that hold those four weights.
 __global__ void debug_indices_kernel(const uint8_t *__restrict__ packed, uint8_t *__restrict__ idx,
                                      uint32_t *status, int K, int N, int bits, int group)
 {
@@ -162,8 +163,12 @@ __global__ void debug_indices_kernel(const uint8_t *__restrict__ packed, uint8_t
     int i = (int)(r / (K / 32));
     uint32_t w = planes[(((size_t)(n >> 2) * bits + i) * (K / 32) + v) * 4 + (n & 3)];
 #pragma unroll
-    for (int e = 0; e < 8; ++e)
-        idx[((size_t)i * (K / 4) + 8 * v + e) * N + n] = (uint8_t)((w >> (4 * e)) & 0xF);
+    for (int e = 0; e < 8; ++e) {
+        uint32_t x = 0;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) x |= ((w >> plane_bit(4 * e + jj)) & 1u) << jj;
+        idx[((size_t)i * (K / 4) + 8 * v + e) * N + n] = (uint8_t)x;
+    }
 }
 
 tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int group, uint8_t *idx,

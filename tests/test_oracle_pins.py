@@ -87,9 +87,22 @@ def test_pack_every_code_value_roundtrips():
         assert np.array_equal(q, codes) and np.array_equal(z, zeros)
 
 
-def test_packed_plane_word_is_a_plain_bit_plane():
+def plane_bit(r):
+    """Bit of a plane word that holds the weight with k % 32 == r (format description: weight
+    8*ph + j sits at bit 4*j + ph)."""
+    return 4 * (r & 7) + (r >> 3)
+
+
+def test_plane_bit_is_a_permutation_of_the_word():
+    assert sorted(plane_bit(r) for r in range(32)) == list(range(32))
+    # nibble j of a word holds the weights j, 8 + j, 16 + j, 24 + j, lowest first
+    for j in range(8):
+        assert [plane_bit(8 * ph + j) for ph in range(4)] == [4 * j + ph for ph in range(4)]
+
+
+def test_packed_plane_word_is_a_permuted_bit_plane():
     # a single set bit lands where the format description says: word (strip nb, plane i,
-    # v = k/32, c = n%4), bit k%32; planes start at byte 256.
+    # v = k/32, c = n%4), bit plane_bit(k%32); planes start at byte 256.
     K, N, G, bits = 128, 8, 32, 3
     for (k, n, code) in [(0, 0, 1), (37, 5, 4), (127, 7, 2), (64, 3, 7)]:
         codes = np.zeros((K, N), dtype=np.uint8)
@@ -100,12 +113,13 @@ def test_packed_plane_word_is_a_plain_bit_plane():
         want = np.zeros_like(words)
         for i in range(bits):
             if (code >> i) & 1:
-                want[(((n // 4) * bits + i) * (K // 32) + k // 32) * 4 + n % 4] = 1 << (k % 32)
+                want[(((n // 4) * bits + i) * (K // 32) + k // 32) * 4 + n % 4] = 1 << plane_bit(k % 32)
         assert np.array_equal(words, want)
 
 
-def test_packed_indices_are_nibbles_of_plane_words():
-    # the 4-bit index idx_i[t, n] is nibble t%8 of the plane word (i, t/8, n)
+def test_packed_indices_can_be_read_out_of_plane_words():
+    # bit j of the 4-bit index idx_i[t, n] (activations 4t .. 4t+3) is bit plane_bit(4*(t%8) + j) of
+    # the plane word (i, t/8, n)
     c = rand_case(1, 128, 8, 4, 32, seed=3)
     idx = orc.indices(c.codes, 4)
     packed = orc.pack(c.codes, c.scales, c.zeros, 4, 32)
@@ -114,7 +128,8 @@ def test_packed_indices_are_nibbles_of_plane_words():
         for t in range(32):
             for n in range(8):
                 w = int(words[(((n // 4) * 4 + i) * 4 + t // 8) * 4 + n % 4])
-                assert (w >> (4 * (t % 8))) & 0xF == idx[i, t, n]
+                got = sum(((w >> plane_bit(4 * (t % 8) + j)) & 1) << j for j in range(4))
+                assert got == idx[i, t, n]
 
 
 # ---- P3, P10: exact zeros --------------------------------------------------
