@@ -318,10 +318,10 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 // the c-th pair of each quarter of the word
                 float xv[8];
 #pragma unroll
-                for (int ph = 0; ph < 4; ++ph) {
-                    const float2 f = __half22float2(reinterpret_cast<const __half2 *>(&xraw[ph])[c]);
-                    xv[ph] = f.x;
-                    xv[ph + 4] = f.y;
+                for (int qq = 0; qq < 4; ++qq) {
+                    const float2 f = __half22float2(reinterpret_cast<const __half2 *>(&xraw[qq])[c]);
+                    xv[qq] = f.x;
+                    xv[qq + 4] = f.y;
                 }
                 float lo[16];
                 lut16(xv[0], xv[1], xv[2], xv[3], lo);
