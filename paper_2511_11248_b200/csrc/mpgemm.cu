@@ -64,6 +64,7 @@ struct GemmParams {
     int sms;
     int R;          // column ranges per row tile
     int wide;       // tile configuration
+    int pair;       // CTA-pair kernel
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -109,6 +110,63 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
             else if (now - t0 > 1000000000ull) return false;
         }
     }
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// Arrive on a barrier of another CTA of the cluster.  Only the signal crosses CTAs: the data a
+// CTA's tensor core reads is in that CTA's own shared memory, made visible by the writer's
+// fence.proxy.async, so no cluster-scope release (a slow memory barrier) is needed here.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_shared_cluster_u32(uint32_t cluster_addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void tcgen05_alloc2(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_relinquish2()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_dealloc2(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// commit of the pair's MMAs, arriving on the barrier at the same address in both CTAs
+__device__ __forceinline__ void tcgen05_commit2_both(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma2_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void fence_barrier_init()
 {
@@ -288,12 +346,13 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
 struct SubTile { int tile_m, col0, bn; };
 
 struct TileWalk {
-    int item, nitems, stride, tiles_m, R, n16, max16;
+    int item, nitems, stride, tiles_m, R, n16, max16, unit;
     int tm, lo, len, nsub, j;
-    __device__ TileWalk(const GemmParams &p, int cta, int ncta, int bn_max)
+    // unit: column granularity (16; 32 for CTA pairs, whose two CTAs each take half of a sub-tile)
+    __device__ TileWalk(const GemmParams &p, int cta, int ncta, int bn_max, int unit_ = 16)
         : item(cta - ncta), nitems(p.tiles_m * p.R), stride(ncta), tiles_m(p.tiles_m), R(p.R),
-          n16((p.N + 15) >> 4),   // a last unit may reach 8 columns past N: computed, never stored
-          max16(bn_max / 16),
+          n16((p.N + unit_ - 1) / unit_),   // a last unit may reach past N: computed, never stored
+          max16(bn_max / unit_), unit(unit_),
           tm(0), lo(0), len(0), nsub(0), j(0) {}
     __device__ bool next(SubTile &t)
     {
@@ -309,8 +368,8 @@ struct TileWalk {
         }
         const int u0 = lo + (len * j) / nsub, u1 = lo + (len * (j + 1)) / nsub;
         t.tile_m = tm;
-        t.col0 = u0 * 16;
-        t.bn = (u1 - u0) * 16;
+        t.col0 = u0 * unit;
+        t.bn = (u1 - u0) * unit;
         ++j;
         return true;
     }
@@ -555,6 +614,259 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     }
 }
 
+// ---- CTA-pair variant ------------------------------------------------------------------------
+// Two CTAs of a cluster share one tile of 2*128*MH tokens x up to 256 output channels: each holds its
+// own 128*MH token rows, dequantizes half of the tile's channels, and the pair multiplies with
+// tcgen05.mma.cta_group::2 (M = 256), issued by the pair's first CTA.  Each SM then reads only half of
+// the weight tile per MMA and dequantizes half as much per flop, which is what the single-CTA kernel
+// is short of (shared-memory bandwidth, ALU pipe).  Barriers that both CTAs feed (weight tile ready,
+// accumulator drained) live in the first CTA and are reached with cluster-scope arrives; the MMA's
+// commits arrive in both CTAs.  No TMA multicast is used: each CTA loads its own tiles.
+constexpr int PAIR_BN = 256;                     // channels of a pair tile (128 per CTA)
+constexpr int PAIR_NSTAGE = 4;
+constexpr int PAIR_B_STAGE_BYTES = (PAIR_BN / 2) * BK * 2;
+constexpr int PAIR_P_PLANE_BYTES = (PAIR_BN / 8) * (BK / 32) * 16;
+constexpr int pair_smem_bytes(int mh, int bits)
+{
+    return PAIR_NSTAGE * (mh * A_HALF_BYTES + PAIR_B_STAGE_BYTES + bits * PAIR_P_PLANE_BYTES) + 1024 + 256;
+}
+
+template <int BITS, int MH>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const GemmParams p)
+{
+    constexpr int NSTAGE = PAIR_NSTAGE, B_STAGE_BYTES = PAIR_B_STAGE_BYTES, P_PLANE_BYTES = PAIR_P_PLANE_BYTES;
+    constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
+    constexpr int P_STAGE_BYTES = BITS * P_PLANE_BYTES;
+    constexpr int TMEM_COLS = MH * PAIR_BN;            // MH accumulators of 256 columns (512 for MH = 2)
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t rank = cluster_ctarank();           // 0: issues the MMAs and owns the shared barriers
+    const bool hdr_ok = header_matches(p.packed, p.K, p.N, p.bits, p.group);   // same answer in every CTA
+    if (!hdr_ok) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
+        return;
+    }
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *a_tiles = smem;
+    uint8_t *b_tiles = smem + NSTAGE * A_STAGE_BYTES;
+    uint8_t *p_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + P_STAGE_BYTES));
+    // bars[0..NSTAGE) loaded (own TMA), [NSTAGE..2NSTAGE) full (both CTAs' dequantization warps; used in
+    // CTA 0), [2NSTAGE..3NSTAGE) empty (MMA commit, both CTAs), then accumulator full (commit, both CTAs)
+    // and accumulator empty (both CTAs' epilogue warps; used in CTA 0)
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * NSTAGE + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_kb = p.K / BK;
+    const uint32_t loaded0 = smem_u32(bars), full0 = smem_u32(bars + NSTAGE), empty0 = smem_u32(bars + 2 * NSTAGE),
+                   accf = smem_u32(bars + 3 * NSTAGE), acce = smem_u32(bars + 3 * NSTAGE + 1);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NSTAGE; ++s) {
+            mbar_init(loaded0 + 8 * s, 1);
+            mbar_init(full0 + 8 * s, 2 * NUM_DEQ_WARPS);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accf, 1);
+        mbar_init(acce, 2 * NUM_EPI_WARPS);
+        *tmem_slot = 0xFFFFFFFFu;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_alloc2(smem_u32(tmem_slot), TMEM_COLS);
+        tcgen05_relinquish2();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                // both CTAs' barriers and tensor memory are set up
+    tcgen05_fence_after();
+    uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
+    if (tmem_base == 0xFFFFFFFFu) tmem_base = ld_shared_cluster_u32(mapa_u32(smem_u32(tmem_slot), rank ^ 1u));
+
+    bool ok = tmem_base != 0xFFFFFFFFu;
+    // the pair walks through its items together; a CTA's rows and channels inside a sub-tile:
+    TileWalk walk(p, (int)(blockIdx.x >> 1), (int)(gridDim.x >> 1), PAIR_BN, 32);
+    SubTile t;
+    const uint32_t full_lead = mapa_u32(full0, 0), acce_lead = mapa_u32(acce, 0);
+    if (warp == 0) {
+        // ---- stage 1: this CTA's activation rows and packed channels by TMA ---------------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            while (ok && walk.next(t)) {
+                const int row0 = t.tile_m * (2 * BM * MH) + (int)rank * (BM * MH);
+                const int strip0 = (t.col0 + (int)rank * (t.bn / 2)) / 4;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % NSTAGE);
+                    const uint32_t ph = (it / NSTAGE) & 1u;
+                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
+                    mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + P_STAGE_BYTES);
+                    tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, row0, loaded0 + 8 * s);
+#pragma unroll
+                    for (int i = 0; i < BITS; ++i)
+                        tma_load_3d(smem_u32(p_tiles + s * P_STAGE_BYTES + i * P_PLANE_BYTES), &tmap_w, kb * (BK / 8), i,
+                                    strip0, loaded0 + 8 * s);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- stage 3: the pair's MMAs, issued by CTA 0 ------------------------------------------
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, ti = 0;
+            while (ok && walk.next(t)) {
+                if (!mbar_wait(acce, (ti & 1u) ^ 1u)) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint32_t idesc = (1u << 4) | ((uint32_t)(t.bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % NSTAGE);
+                    const uint32_t ph = (it / NSTAGE) & 1u;
+                    if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
+#pragma unroll
+                    for (int j = 0; j < BK / 16; ++j)
+#pragma unroll
+                        for (int h = 0; h < MH; ++h) {
+                            const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES + h * A_HALF_BYTES));
+                            tcgen05_mma2_f16(tmem_base + (uint32_t)(h * PAIR_BN), adesc + 2 * j, bdesc + 2 * j, idesc,
+                                             (kb > 0 || j > 0) ? 1u : 0u);
+                        }
+                    tcgen05_commit2_both(empty0 + 8 * s);
+                }
+                if (ok) tcgen05_commit2_both(accf);
+                ++ti;
+            }
+        }
+    } else if (warp < 2 + NUM_DEQ_WARPS) {
+        // ---- stage 2: two-level lookup dequantization of this CTA's half of the channels --------
+        // at most 128 channels per CTA: the two halves of the sixteen warps take turns, two k-blocks each
+        const int wd16 = warp - 2;
+        const int wd = wd16 & (NUM_DEQ_WARPS / 2 - 1), grp = wd16 / (NUM_DEQ_WARPS / 2);
+        const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
+        const int nblk = p.K / p.group;
+        const int gshift = (p.group == 32) ? 5 : (p.group == 64) ? 6 : 7;
+        auto block_of = [&](int kb) { return ((2 * kb + v) * 32) >> gshift; };
+        const int n_local = wd * 16 + sl * 4 + c;
+        const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
+        const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
+        const uint32_t xr = (uint32_t)(n_local & 7);
+        const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
+        auto mine = [&](int kb) { return ((kb >> 1) & 1) == grp; };
+        auto next_mine = [&](int kb) { return !(kb & 1) ? kb + 1 : kb + 3; };
+
+        uint32_t it0 = 0;
+        while (ok && walk.next(t)) {
+            const int half = t.bn / 2;
+            const int n = t.col0 + (int)rank * half + n_local;
+            const bool valid = n_local < half && n < p.N;
+            const int nb = n >> 2;
+            const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
+            const uint16_t *pz = p.zeros + (size_t)nb * nblk;
+            auto fetch_sz = [&](int B, __half &sv, uint32_t &zz) {
+                sv = __float2half(0.f);
+                zz = 0u;
+                if (valid && B < nblk) {
+                    sv = __ldg(ps + (size_t)B * 4);
+                    zz = ((uint32_t)__ldg(pz + B) >> (4 * c)) & 0xFu;
+                }
+            };
+            ConvTable<BITS> T;
+            int cur_B = -1, next_B = -1;
+            __half sv_next = __float2half(0.f);
+            uint32_t zz_next = 0u;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const uint32_t it = it0 + (uint32_t)kb;
+                const int s = (int)(it % NSTAGE);
+                const uint32_t ph = (it / NSTAGE) & 1u;
+                const bool work = valid && mine(kb);
+                if (work) {
+                    const int Bk = block_of(kb);
+                    if (Bk != cur_B) {
+                        if (next_B != Bk) fetch_sz(Bk, sv_next, zz_next);
+                        cur_B = Bk;
+                        T.build(sv_next, zz_next);
+                    }
+                    const int kn = next_mine(kb);
+                    const int Bn = block_of(kn);
+                    if (kn < num_kb && Bn != cur_B && Bn != next_B) {
+                        next_B = Bn;
+                        fetch_sz(Bn, sv_next, zz_next);
+                    }
+                }
+                if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
+                if (work) {
+                    uint32_t w[BITS];
+                    const uint32_t pp = p_base + (uint32_t)s * P_STAGE_BYTES;
+#pragma unroll
+                    for (int i = 0; i < BITS; ++i)
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[i]) : "r"(pp + i * P_PLANE_BYTES) : "memory");
+                    uint32_t out[16];
+                    dequant_word<BITS>(w, T, out);
+                    const uint32_t row = b_base + (uint32_t)s * B_STAGE_BYTES;
+#pragma unroll
+                    for (int cj = 0; cj < 4; ++cj) {
+                        const uint32_t chunk = ((uint32_t)(4 * v + cj)) ^ xr;
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(row + chunk * 16u), "r"(out[4 * cj]),
+                                     "r"(out[4 * cj + 1]), "r"(out[4 * cj + 2]), "r"(out[4 * cj + 3]) : "memory");
+                    }
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(full_lead + 8 * s);
+            }
+            it0 += (uint32_t)num_kb;
+        }
+    } else {
+        // ---- epilogue: this CTA's rows, tensor memory -> fp16 -> global -----------------------------
+        const int quarter = warp & 3;
+        const int epart = (warp - 2 - NUM_DEQ_WARPS) >> 2;
+        uint32_t ti = 0;
+        while (ok && walk.next(t)) {
+            if (!mbar_wait(accf, ti & 1u)) { ok = false; break; }
+            tcgen05_fence_after();
+#pragma unroll 1
+            for (int h = 0; h < MH; ++h) {
+                const int m = t.tile_m * (2 * BM * MH) + (int)rank * (BM * MH) + h * BM + quarter * 32 + lane;
+#pragma unroll 1
+                for (int col = 32 * epart; col < t.bn; col += 32 * (NUM_EPI_WARPS / 4)) {
+                    uint32_t r[32];
+                    tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * PAIR_BN + col), r);
+                    tcgen05_wait_ld();
+                    if (m < p.M) {
+                        __half *dst = p.y + (size_t)m * p.N + (size_t)t.col0 + col;
+#pragma unroll
+                        for (int g8 = 0; g8 < 4; ++g8) {
+                            if (col + 8 * g8 < t.bn && t.col0 + col + 8 * g8 < p.N) {
+                                uint32_t hv[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __half2 hh = __floats2half2_rn(__uint_as_float(r[8 * g8 + 2 * e]),
+                                                                         __uint_as_float(r[8 * g8 + 2 * e + 1]));
+                                    hv[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + 8 * g8) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
+                            }
+                        }
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acce_lead);
+            ++ti;
+        }
+    }
+
+    if (!ok) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                // nobody touches the peer's memory after this
+    if (warp == 1 && tmem_base != 0xFFFFFFFFu) {
+        tcgen05_fence_after();
+        tcgen05_dealloc2(tmem_base, TMEM_COLS);
+    }
+}
+
 // ---- host side ---------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -583,9 +895,34 @@ tman_status launch_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, co
     return launch_status();
 }
 
+template <int BITS, int MH>
+tman_status launch_pair_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, cudaStream_t s)
+{
+    auto kern = mpgemm_pair_kernel<BITS, MH>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pair_smem_bytes(MH, BITS)) != cudaSuccess)
+        return TMAN_ERR_CUDA;
+    long long pairs = p.sms / 2;
+    if (pairs > (long long)p.tiles_m * p.R) pairs = (long long)p.tiles_m * p.R;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = pair_smem_bytes(MH, BITS);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, p) != cudaSuccess) return TMAN_ERR_CUDA;
+    return TMAN_OK;
+}
+
 template <int BITS>
 tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, int mh, cudaStream_t s)
 {
+    if (p.pair) return mh == 2 ? launch_pair_tile<BITS, 2>(tmap_x, tmap_w, p, s) : launch_pair_tile<BITS, 1>(tmap_x, tmap_w, p, s);
     if (p.wide) return mh == 2 ? launch_tile<BITS, 2, 1>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 1>(tmap_x, tmap_w, p, s);
     return mh == 2 ? launch_tile<BITS, 2, 0>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 0>(tmap_x, tmap_w, p, s);
 }
@@ -603,6 +940,13 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     CUtensorMap tmap;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    // CTA pairs (each CTA 256 token rows of a 512-row tile, half of the tile's channels) when there
+    // are enough tokens and a pair of SMs gets a share of the output at least 192 channels wide;
+    // otherwise single CTAs, which waste less on narrow shares.
+    const int sms_q = sm_count();
+    if (sms_q <= 0) return TMAN_ERR_CUDA;
+    const long long share = (long long)N * ((M + 4 * BM - 1) / (4 * BM)) / (sms_q / 2 > 0 ? sms_q / 2 : 1);
+    const bool pair = M > 2 * BM && share >= 192;
     const int mh = (M > BM) ? 2 : 1;                   // row blocks per CTA
     const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)(BM * mh)};
     const cuuint32_t estr[2] = {1, 1};
@@ -621,14 +965,29 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.y = static_cast<__half *>(y);
     p.status = static_cast<uint32_t *>(ws);
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
-    p.tiles_m = (M + BM * mh - 1) / (BM * mh);
+    p.pair = pair ? 1 : 0;
+    p.tiles_m = pair ? (M + 2 * BM * mh - 1) / (2 * BM * mh) : (M + BM * mh - 1) / (BM * mh);
     p.sms = sm_count();
     if (p.sms <= 0) return TMAN_ERR_CUDA;
     // Tile configuration and column ranges per row tile: the pair that minimises (waves of items over
     // the SMs) x (cost of an item).  A sub-tile of w 16-column units costs about w + 10 units of
     // shared-memory traffic per k-block (the activation tile is written once and read once per MMA
     // whatever the width), and a wide sub-tile holds twice as many units as a narrow one.
-    {
+    if (pair) {
+        // pairs: units of 32 columns, sub-tiles of up to 8 units, one item at a time per pair of SMs
+        const int n32 = (N + 31) / 32, npairs = p.sms / 2;
+        double best = 1e300;
+        p.R = 1;
+        p.wide = 0;
+        for (int R = 1; R <= n32 && R <= 4096; ++R) {
+            const long long items = (long long)p.tiles_m * R;
+            const long long waves = (items + npairs - 1) / npairs;
+            const int w = (n32 + R - 1) / R;
+            const int nsub = (w + 7) / 8;
+            const double cost = (double)waves * (w + 3.0 * nsub);
+            if (cost < best - 1e-9) { best = cost; p.R = R; }
+        }
+    } else {
         const int n16 = (N + 15) / 16;
         double best = 1e300;
         p.R = 1;
@@ -652,7 +1011,7 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
         const cuuint64_t wt = (cuuint64_t)(K / 32);
         const cuuint64_t wdims[3] = {wt * 4, (cuuint64_t)bits, (cuuint64_t)(N / 4)};
         const cuuint64_t wstrides[2] = {wt * 16, wt * 16 * (cuuint64_t)bits};
-        const cuuint32_t wbox[3] = {(cuuint32_t)(BK / 8), 1, (cuuint32_t)((p.wide ? Cfg<1>::BN : Cfg<0>::BN) / 4)};
+        const cuuint32_t wbox[3] = {(cuuint32_t)(BK / 8), 1, (cuuint32_t)((pair ? PAIR_BN / 2 : (p.wide ? Cfg<1>::BN : Cfg<0>::BN)) / 4)};
         const cuuint32_t westr[3] = {1, 1, 1};
         if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t *>(pk + L.planes_off), wdims, wstrides,
                 wbox, westr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,

@@ -53,6 +53,17 @@ def test_small_cases(M, K, N, bits, G):
     check_full(synth.small_case(M, K, N, bits, G, seed=M + K + N + bits, outliers=(bits == 4)))
 
 
+# Enough tokens and channels for the CTA-pair kernel (512-row tiles split over two SMs), with ragged
+# row tiles, ragged channel ranges and every bit width; compared element by element.
+PAIRED = [(600, 256, 7176, 2, 64), (1030, 128, 4744, 3, 128), (513, 192, 14344, 4, 64),
+          (1024, 320, 3560, 4, 32)]
+
+
+@pytest.mark.parametrize("M,K,N,bits,G", PAIRED)
+def test_pair_kernel_cases(M, K, N, bits, G):
+    check_full(synth.small_case(M, K, N, bits, G, seed=M + K + N + bits, outliers=(bits == 4)))
+
+
 def test_integer_case_is_exact():
     rng = np.random.default_rng(5)
     c = synth.small_case(130, 512, 136, 3, 64, seed=31)
