@@ -188,6 +188,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tma
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
+// Tile store: shared memory (written by this warp, made visible with fence.proxy.async) -> global.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *tmap, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(src) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the issuing thread's earlier tile stores have finished reading shared memory / have completed
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_alloc(uint32_t dst_smem, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -626,14 +636,18 @@ constexpr int PAIR_BN = 256;                     // channels of a pair tile (128
 constexpr int PAIR_NSTAGE = 4;
 constexpr int PAIR_B_STAGE_BYTES = (PAIR_BN / 2) * BK * 2;
 constexpr int PAIR_P_PLANE_BYTES = (PAIR_BN / 8) * (BK / 32) * 16;
+constexpr int PAIR_OUT_BYTES = 32 * 32 * 2;      // an epilogue warp's output staging: 32 tokens x 32 channels
 constexpr int pair_smem_bytes(int mh, int bits)
 {
-    return PAIR_NSTAGE * (mh * A_HALF_BYTES + PAIR_B_STAGE_BYTES + bits * PAIR_P_PLANE_BYTES) + 1024 + 256;
+    // stages, barriers (256 B), staging (1024-aligned as the stages are: bits * 1 KB keeps it so), slack to align
+    return PAIR_NSTAGE * (mh * A_HALF_BYTES + PAIR_B_STAGE_BYTES + bits * PAIR_P_PLANE_BYTES) + 1024
+           + NUM_EPI_WARPS * PAIR_OUT_BYTES + 256;
 }
 
 template <int BITS, int MH>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const GemmParams p)
+mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                   const __grid_constant__ CUtensorMap tmap_y, const GemmParams p)
 {
     constexpr int NSTAGE = PAIR_NSTAGE, B_STAGE_BYTES = PAIR_B_STAGE_BYTES, P_PLANE_BYTES = PAIR_P_PLANE_BYTES;
     constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
@@ -650,7 +664,8 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     uint8_t *a_tiles = smem;
     uint8_t *b_tiles = smem + NSTAGE * A_STAGE_BYTES;
     uint8_t *p_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + P_STAGE_BYTES));
+    uint8_t *out_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + P_STAGE_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(out_tiles + NUM_EPI_WARPS * PAIR_OUT_BYTES);
     // bars[0..NSTAGE) loaded (own TMA), [NSTAGE..2NSTAGE) full (both CTAs' dequantization warps; used in
     // CTA 0), [2NSTAGE..3NSTAGE) empty (MMA commit, both CTAs), then accumulator full (commit, both CTAs)
     // and accumulator empty (both CTAs' epilogue warps; used in CTA 0)
@@ -817,44 +832,63 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             it0 += (uint32_t)num_kb;
         }
     } else {
-        // ---- epilogue: this CTA's rows, tensor memory -> fp16 -> global -----------------------------
+        // ---- epilogue: this CTA's rows, tensor memory -> fp16 -> shared memory -> global (tile stores) --
+        // A warp reads 32 tokens x 32 channels (one token per lane), writes them as 64-byte rows into its
+        // staging tile in the 64-byte swizzle (16-byte chunk index ^ bits 1..2 of the row: no bank
+        // conflicts) and one lane stores the tile; tokens >= M and channels >= N are clipped by the store.
         const int quarter = warp & 3;
-        const int epart = (warp - 2 - NUM_DEQ_WARPS) >> 2;
+        const int ew = warp - 2 - NUM_DEQ_WARPS, epart = ew >> 2;
+        const uint32_t stage = smem_u32(out_tiles + ew * PAIR_OUT_BYTES);
+        const uint32_t my_row = stage + (uint32_t)lane * 64u, xr = ((uint32_t)lane >> 1) & 3u;
         uint32_t ti = 0;
         while (ok && walk.next(t)) {
             if (!mbar_wait(accf, ti & 1u)) { ok = false; break; }
             tcgen05_fence_after();
+            bool released = false;
 #pragma unroll 1
             for (int h = 0; h < MH; ++h) {
-                const int m = t.tile_m * (2 * BM * MH) + (int)rank * (BM * MH) + h * BM + quarter * 32 + lane;
+                const int m0 = t.tile_m * (2 * BM * MH) + (int)rank * (BM * MH) + h * BM + quarter * 32;
 #pragma unroll 1
                 for (int col = 32 * epart; col < t.bn; col += 32 * (NUM_EPI_WARPS / 4)) {
+                    const bool last = (h == MH - 1) && (col + 32 * (NUM_EPI_WARPS / 4) >= t.bn);
                     uint32_t r[32];
-                    tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * PAIR_BN + col), r);
-                    tcgen05_wait_ld();
-                    if (m < p.M) {
-                        __half *dst = p.y + (size_t)m * p.N + (size_t)t.col0 + col;
+                    if (m0 < p.M) {
+                        tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * PAIR_BN + col), r);
+                        tcgen05_wait_ld();
+                    }
+                    if (last) {                        // the accumulators are read: the next tile's MMAs may start
+                        tcgen05_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(acce_lead);
+                        released = true;
+                    }
+                    if (m0 < p.M) {
+                        uint32_t hv[16];
 #pragma unroll
-                        for (int g8 = 0; g8 < 4; ++g8) {
-                            if (col + 8 * g8 < t.bn && t.col0 + col + 8 * g8 < p.N) {
-                                uint32_t hv[4];
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const __half2 hh = __floats2half2_rn(__uint_as_float(r[8 * g8 + 2 * e]),
-                                                                         __uint_as_float(r[8 * g8 + 2 * e + 1]));
-                                    hv[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                                }
-                                *reinterpret_cast<uint4 *>(dst + 8 * g8) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
-                            }
+                        for (int e = 0; e < 16; ++e) {
+                            const __half2 hh = __floats2half2_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                            hv[e] = *reinterpret_cast<const uint32_t *>(&hh);
                         }
+                        if (lane == 0) tma_store_wait_read();      // the staging tile is free again
+                        __syncwarp();
+#pragma unroll
+                        for (uint32_t cj = 0; cj < 4; ++cj)
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((cj ^ xr) << 4)), "r"(hv[4 * cj]),
+                                         "r"(hv[4 * cj + 1]), "r"(hv[4 * cj + 2]), "r"(hv[4 * cj + 3]) : "memory");
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) tma_store_2d(&tmap_y, stage, t.col0 + col, m0);
                     }
                 }
             }
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(acce_lead);
+            if (!released) {                           // a warp without a chunk in this sub-tile
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(acce_lead);
+            }
             ++ti;
         }
+        if (lane == 0) tma_store_wait_all();
     }
 
     if (!ok) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
@@ -896,7 +930,8 @@ tman_status launch_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, co
 }
 
 template <int BITS, int MH>
-tman_status launch_pair_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, cudaStream_t s)
+tman_status launch_pair_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y,
+                             const GemmParams &p, cudaStream_t s)
 {
     auto kern = mpgemm_pair_kernel<BITS, MH>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pair_smem_bytes(MH, BITS)) != cudaSuccess)
@@ -915,14 +950,15 @@ tman_status launch_pair_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, p) != cudaSuccess) return TMAN_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, p) != cudaSuccess) return TMAN_ERR_CUDA;
     return TMAN_OK;
 }
 
 template <int BITS>
-tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, int mh, cudaStream_t s)
+tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y,
+                        const GemmParams &p, int mh, cudaStream_t s)
 {
-    if (p.pair) return mh == 2 ? launch_pair_tile<BITS, 2>(tmap_x, tmap_w, p, s) : launch_pair_tile<BITS, 1>(tmap_x, tmap_w, p, s);
+    if (p.pair) return launch_pair_tile<BITS, 2>(tmap_x, tmap_w, tmap_y, p, s);   // pairs run on more than 256 tokens
     if (p.wide) return mh == 2 ? launch_tile<BITS, 2, 1>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 1>(tmap_x, tmap_w, p, s);
     return mh == 2 ? launch_tile<BITS, 2, 0>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 0>(tmap_x, tmap_w, p, s);
 }
@@ -1018,9 +1054,19 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return TMAN_ERR_CUDA;
     }
-    if (bits == 2) return launch_bits<2>(tmap, tmap_w, p, mh, s);
-    if (bits == 3) return launch_bits<3>(tmap, tmap_w, p, mh, s);
-    return launch_bits<4>(tmap, tmap_w, p, mh, s);
+    // the output as 32 x 32 tiles in the 64-byte swizzle (the pair kernel's epilogue stores)
+    CUtensorMap tmap_y;
+    {
+        const cuuint64_t ydims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+        const cuuint64_t ystrides[1] = {(cuuint64_t)N * 2};
+        const cuuint32_t ybox[2] = {32, 32};
+        if (enc(&tmap_y, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, ydims, ystrides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TMAN_ERR_CUDA;
+    }
+    if (bits == 2) return launch_bits<2>(tmap, tmap_w, tmap_y, p, mh, s);
+    if (bits == 3) return launch_bits<3>(tmap, tmap_w, tmap_y, p, mh, s);
+    return launch_bits<4>(tmap, tmap_w, tmap_y, p, mh, s);
 }
 
 }  // namespace tman

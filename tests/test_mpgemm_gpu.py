@@ -55,8 +55,8 @@ def test_small_cases(M, K, N, bits, G):
 
 # Enough tokens and channels for the CTA-pair kernel (512-row tiles split over two SMs), with ragged
 # row tiles, ragged channel ranges and every bit width; compared element by element.
-PAIRED = [(600, 256, 7176, 2, 64), (1030, 128, 4744, 3, 128), (513, 192, 14344, 4, 64),
-          (1024, 320, 3560, 4, 32)]
+PAIRED = [(600, 256, 7176, 2, 64), (1030, 128, 4744, 3, 128), (513, 256, 14344, 4, 64),
+          (1024, 384, 3560, 4, 32)]
 
 
 @pytest.mark.parametrize("M,K,N,bits,G", PAIRED)
