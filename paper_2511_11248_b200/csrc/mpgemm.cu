@@ -2,22 +2,29 @@
 // (paper Sec. 4.1 "Unified Layout through Fused LUT-based Dequantization", Fig. 7;
 //  Sec. 4.2 "Pipelining to Hide Dequantization Overhead", Fig. 9).
 //
-// A CTA computes tiles of 128*MH tokens x up to 128 output channels, one after the other (one CTA per
-// SM, each with an equal share of the output).  Four kinds of agents run concurrently on a ring of
-// shared-memory stages guarded by mbarriers (the paper's DMA / vector-core / matrix-core stages):
+// The output is cut into tiles of 256 channels x 128*MH tokens (one CTA, at most 128 tokens) or
+// 256*MH tokens (a pair of CTAs on two SMs).  A tile's work is its K/64 k-blocks; the k-blocks of all
+// tiles, laid end to end, are dealt to the workers (CTAs or pairs, one per SM or SM pair) in equal
+// contiguous spans, so every SM is busy to the end whatever the shape.  A tile whose k-blocks fall
+// into several spans is summed through fp32 partial tiles in the workspace (see "split tiles").
+// Four kinds of agents run concurrently on a ring of shared-memory stages guarded by mbarriers (the
+// paper's DMA / vector-core / matrix-core stages):
 //   * warp 0, one lane : TMA loads of the fp16 activation tile (128-byte swizzle) and of the packed
 //                        bit-plane words of the weight tile (one box per plane);
-//   * warps 2..17      : (two groups of eight that take turns, two k-blocks each) read the staged
-//                        plane words of their column, rebuild the codes
+//   * warps 2..17      : read the staged plane words of their column, rebuild the codes
 //                        (level 1: bit-serial -> bit-parallel), look every code up in the
 //                        per-(block, column) conversion table kept in registers and addressed
 //                        with byte-permute instructions (level 2: scale and zero-point baked in),
 //                        and write the fp16 weight tile in the K-major swizzled layout the
 //                        tensor core reads;
-//   * warp 1, one lane : tcgen05.mma (M128 N<=128 K16, fp16 x fp16 -> fp32 in tensor memory), one
-//                        per row block; tcgen05.commit hands the stage back;
-//   * warps 18..25     : epilogue of the previous tile (tcgen05.ld, round to fp16, store) while the
-//                        next tile accumulates into the second set of tensor-memory columns.
+//   * warp 1, one lane : tcgen05.mma (fp16 x fp16 -> fp32 in tensor memory), one per row block and
+//                        16 k; tcgen05.commit hands the stage back;
+//   * warps 18..25     : epilogue (tcgen05.ld, round to fp16, stage in shared memory, TMA tile store).
+// CTA pairs (more than 128 tokens): each CTA holds its own 128*MH token rows and dequantizes half of
+// the tile's channels, and the pair multiplies with tcgen05.mma.cta_group::2 (M = 256), issued by the
+// pair's first CTA: every weight is rebuilt once per 256*MH tokens and each SM reads half of the
+// weight tile per MMA.  Barriers that both CTAs feed (weight tile ready, accumulator drained) live in
+// the first CTA; the MMA's commits arrive in both.  No TMA multicast: each CTA loads its own tiles.
 // Every wait is bounded: when a bound is hit the kernel records TMAN_ERR_TIMEOUT, stops issuing
 // work, and still reaches the common tear-down that frees tensor memory.
 #include "common.cuh"
@@ -27,44 +34,49 @@
 namespace tman {
 namespace {
 
-// A CTA multiplies MH row blocks of 128 tokens by one dequantized weight tile of up to BN columns: every
-// weight is rebuilt once per 128*MH tokens (MH = 2 halves the dequantization work per flop).
-// Two tile configurations.  WIDE: BN = 256, one MMA covers 256 output channels, so an activation tile
-// is read from shared memory once per 256 channels (shared-memory bandwidth is what bounds this
-// kernel); three stages of 72 KB fit and tensor memory holds one accumulator set.  Narrow: BN = 128,
-// four stages and two accumulator sets (the epilogue of a sub-tile overlaps the next one); used when
-// the output is so small that an SM's share is at most 128 columns wide.
-constexpr int BM = 128, BK = 64;
-template <int WIDE> struct Cfg {
-    static constexpr int BN = WIDE ? 256 : 128;
-    static constexpr int NSTAGE = WIDE ? 3 : 4;
-    static constexpr int NACC = WIDE ? 1 : 2;       // accumulator sets in tensor memory (MH * BN columns each)
-    static constexpr int B_STAGE_BYTES = BN * BK * 2;
-    static constexpr int P_PLANE_BYTES = (BN / 4) * (BK / 32) * 16;   // one plane of a packed tile
-};
+constexpr int BM = 128, BK = 64, BN = 256;      // token rows of a row block, k-block, channels of a tile
 constexpr int A_HALF_BYTES = BM * BK * 2;
 constexpr int NUM_DEQ_WARPS = 16;               // each fills 16 columns of a weight tile
 constexpr int NUM_EPI_WARPS = 8;                // two per quarter of the tensor-memory lanes (alternate 32-column chunks)
 constexpr int GEMM_THREADS = 32 * (2 + NUM_DEQ_WARPS + NUM_EPI_WARPS);
-template <int WIDE> constexpr int smem_bytes(int mh, int bits)
-{
-    return Cfg<WIDE>::NSTAGE * (mh * A_HALF_BYTES + Cfg<WIDE>::B_STAGE_BYTES + bits * Cfg<WIDE>::P_PLANE_BYTES) +
-           1024 /*align*/ + 256 /*barriers*/;
-}
+constexpr int OUT_TILE_BYTES = 32 * 32 * 2;     // an epilogue warp's output staging: 32 tokens x 32 channels
+constexpr int CHUNK_BYTES = 32 * 32 * 4;        // the same chunk as fp32 partial sums
+constexpr int PART_RING = 4;                    // partial chunks an epilogue warp keeps in flight when it sums a split tile
+constexpr int kMaxGemmCtas = 160;               // the workspace is sized for at most this many CTAs
+
+template <int MH, bool PAIR> struct Cfg {
+    static constexpr int NCTA = PAIR ? 2 : 1;
+    static constexpr int BN_CTA = BN / NCTA;                          // channels a CTA dequantizes
+    static constexpr int NSTAGE = PAIR ? 4 : 3;
+    static constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
+    static constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;
+    static constexpr int P_PLANE_BYTES = (BN_CTA / 4) * (BK / 32) * 16;   // one plane of a CTA's packed tile
+    static constexpr int TMEM_COLS = MH * BN;                         // one fp32 accumulator of BN columns per row block
+    static constexpr int smem_bytes(int bits)
+    {
+        // stages (multiples of 1 KB, so the staging tiles stay 1 KB aligned), staging, barriers, slack to align
+        return NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + bits * P_PLANE_BYTES) + NUM_EPI_WARPS * OUT_TILE_BYTES + 512 + 1024;
+    }
+};
+
+// Workspace: status word (kWsStatusBytes), one flag per epilogue warp of every CTA, then one fp32
+// partial tile per CTA (a worker writes at most one per launch).
+constexpr size_t kGemmFlagsOff = kWsStatusBytes;
+constexpr size_t kGemmPartialOff = kWsStatusBytes + 8192;
+constexpr uint32_t kFlagEmpty = 0x7FA5A5A5u;    // what tman_workspace_init leaves behind
+constexpr size_t partial_bytes_per_cta(int mh) { return (size_t)NUM_EPI_WARPS * mh * (BN / 64) * CHUNK_BYTES; }
 
 struct GemmParams {
     const uint8_t  *packed;
     const uint32_t *planes;
     const __half   *scales;
     const uint16_t *zeros;
-    __half         *y;
     uint32_t       *status;
+    uint32_t       *flags;
+    float          *partial;
     int M, K, N, bits, group;
-    int tiles_m;
-    int sms;
-    int R;          // column ranges per row tile
-    int wide;       // tile configuration
-    int pair;       // CTA-pair kernel
+    int tiles_m, tiles_n;
+    int whole_tiles;           // spans are whole tiles (no tile is split)
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -187,6 +199,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tma
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+// Plain bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion on an mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 // Tile store: shared memory (written by this warp, made visible with fence.proxy.async) -> global.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *tmap, uint32_t src, int x, int y)
@@ -349,314 +367,87 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
         }
 }
 
-// Work of a CTA.  The output is cut into row tiles of 128*MH tokens and, inside a row tile, into R
-// column ranges of (almost) equal width, a multiple of 16 columns.  The tiles_m * R items are dealt
-// to the CTAs round-robin; a CTA walks through an item in sub-tiles of at most BN columns, again of
-// (almost) equal width.  Every role derives the same list from (blockIdx, gridDim).
-struct SubTile { int tile_m, col0, bn; };
+// ---- split of the work ----------------------------------------------------------------------
+// T tiles (row tile fastest), W workers.  The first floor(T / W) * W tiles are dealt whole, round-robin.
+// The k-blocks of the remaining tiles (fewer than W), laid end to end in units of two k-blocks (a
+// 128-wide quantization block is never cut), are dealt in equal contiguous spans, so every worker is
+// busy to the end whatever the shape.  A span is shorter than a tile: it is a piece of one tile or the
+// end of one and the start of the next.  A tile cut into several pieces ("split tile") is summed by
+// the worker that owns its last unit: the others, which all have lower numbers, write their fp32
+// accumulators to the workspace and raise a flag.  A worker's walk: first the piece that it only
+// contributes (so that it is ready long before it is needed), then its whole tiles, last the piece
+// of the tile that it finishes.  (whole_tiles: all T tiles are dealt whole.)
+struct Segment { int tile, kb0, kb1; bool whole, finishes; };
 
-struct TileWalk {
-    int item, nitems, stride, tiles_m, R, n16, max16, unit;
-    int tm, lo, len, nsub, j;
-    // unit: column granularity (16; 32 for CTA pairs, whose two CTAs each take half of a sub-tile)
-    __device__ TileWalk(const GemmParams &p, int cta, int ncta, int bn_max, int unit_ = 16)
-        : item(cta - ncta), nitems(p.tiles_m * p.R), stride(ncta), tiles_m(p.tiles_m), R(p.R),
-          n16((p.N + unit_ - 1) / unit_),   // a last unit may reach past N: computed, never stored
-          max16(bn_max / unit_), unit(unit_),
-          tm(0), lo(0), len(0), nsub(0), j(0) {}
-    __device__ bool next(SubTile &t)
+struct Span {
+    long long full, Ur;        // tiles dealt whole; units of the remaining tiles
+    long long next_whole;      // next whole tile of this worker
+    int nu, W, w;
+    int npieces, piece;        // pieces of this worker's span, in walk order, and the next one
+    Segment pieces[3];
+    int first_late;            // pieces[first_late..] come after the whole tiles
+    __device__ Span(const GemmParams &p, int worker, int nworkers)
+        : nu(p.K / (2 * BK)), W(nworkers), w(worker), npieces(0), piece(0), first_late(0)
     {
-        if (j == nsub) {
-            item += stride;
-            if (item >= nitems) return false;
-            tm = item % tiles_m;
-            const int r = item / tiles_m;
-            lo = (int)(((long long)n16 * r) / R);
-            len = (int)(((long long)n16 * (r + 1)) / R) - lo;
-            nsub = (len + max16 - 1) / max16;
-            j = 0;
+        const long long T = (long long)p.tiles_m * p.tiles_n;
+        full = p.whole_tiles ? T : (T / nworkers) * nworkers;
+        Ur = (T - full) * nu;
+        next_whole = worker;
+        long long lo = Ur * worker / nworkers, hi = Ur * (worker + 1) / nworkers;
+        Segment early[3], late[3];
+        int ne = 0, nl = 0;
+        while (hi > lo && ne + nl < 3) {               // from the last tile of the span to the first
+            const long long tile = (hi - 1) / nu, t0 = tile * nu;
+            const long long k0 = (lo > t0) ? lo - t0 : 0, k1 = hi - t0;
+            Segment s;
+            s.tile = (int)(full + tile);
+            s.kb0 = 2 * (int)k0;
+            s.kb1 = 2 * (int)k1;
+            s.whole = (k0 == 0 && k1 == nu);
+            s.finishes = (k1 == nu);
+            if (s.finishes) late[nl++] = s;
+            else early[ne++] = s;
+            hi = t0 + k0;
         }
-        const int u0 = lo + (len * j) / nsub, u1 = lo + (len * (j + 1)) / nsub;
-        t.tile_m = tm;
-        t.col0 = u0 * unit;
-        t.bn = (u1 - u0) * unit;
-        ++j;
-        return true;
+        for (int i = 0; i < ne; ++i) pieces[npieces++] = early[i];
+        first_late = npieces;
+        for (int i = 0; i < nl; ++i) pieces[npieces++] = late[i];   // the tile this worker sums comes last
+    }
+    __device__ bool next(Segment &s)
+    {
+        if (piece < first_late) { s = pieces[piece++]; return true; }
+        if (next_whole < full) {
+            s.tile = (int)next_whole;
+            s.kb0 = 0;
+            s.kb1 = 2 * nu;
+            s.whole = s.finishes = true;
+            next_whole += W;
+            return true;
+        }
+        if (piece < npieces) { s = pieces[piece++]; return true; }
+        return false;
+    }
+    // the worker that owns unit u of tile `tile` (one of the remaining tiles)
+    __device__ int owner(int tile, int u) const
+    {
+        const long long g = (long long)(tile - full) * nu + u;
+        return (int)(((g + 1) * W - 1) / Ur);
     }
 };
 
-template <int BITS, int MH, int WIDE>
+template <int BITS, int MH, bool PAIR>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const GemmParams p)
+mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+              const __grid_constant__ CUtensorMap tmap_y, const GemmParams p)
 {
-    constexpr int BN = Cfg<WIDE>::BN, NSTAGE = Cfg<WIDE>::NSTAGE, NACC = Cfg<WIDE>::NACC;
-    constexpr int B_STAGE_BYTES = Cfg<WIDE>::B_STAGE_BYTES, P_PLANE_BYTES = Cfg<WIDE>::P_PLANE_BYTES;
-    constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
-    constexpr int ACC_COLS = MH * BN;                  // one fp32 accumulator of BN columns per row block
-    constexpr int TMEM_COLS = NACC * ACC_COLS;
-    constexpr int P_STAGE_BYTES = BITS * P_PLANE_BYTES;
+    using C = Cfg<MH, PAIR>;
+    constexpr int NCTA = C::NCTA, NSTAGE = C::NSTAGE, A_STAGE_BYTES = C::A_STAGE_BYTES, B_STAGE_BYTES = C::B_STAGE_BYTES;
+    constexpr int P_PLANE_BYTES = C::P_PLANE_BYTES, P_STAGE_BYTES = BITS * P_PLANE_BYTES, TMEM_COLS = C::TMEM_COLS;
+    constexpr int ROWS_CTA = BM * MH;                  // token rows of a tile held by one CTA
+    constexpr int NGROUP = PAIR ? 2 : 1;               // dequantization warp groups that take turns
     extern __shared__ uint8_t smem_raw[];
-    if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {
-        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
-        return;
-    }
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *a_tiles = smem;
-    uint8_t *b_tiles = smem + NSTAGE * A_STAGE_BYTES;
-    uint8_t *p_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + P_STAGE_BYTES));
-    // bars[0..NSTAGE) loaded (TMA), [NSTAGE..2NSTAGE) full (dequantized), [2NSTAGE..3NSTAGE) empty,
-    // then accumulator full[2], accumulator empty[2]
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * NSTAGE + 4);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_kb = p.K / BK;
-
-    const uint32_t loaded0 = smem_u32(bars), full0 = smem_u32(bars + NSTAGE), empty0 = smem_u32(bars + 2 * NSTAGE),
-                   accf0 = smem_u32(bars + 3 * NSTAGE), acce0 = smem_u32(bars + 3 * NSTAGE + 2);
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < NSTAGE; ++s) {
-            mbar_init(loaded0 + 8 * s, 1);
-            mbar_init(full0 + 8 * s, NUM_DEQ_WARPS);
-            mbar_init(empty0 + 8 * s, 1);
-        }
-        for (int b = 0; b < NACC; ++b) {
-            mbar_init(accf0 + 8 * b, 1);
-            mbar_init(acce0 + 8 * b, NUM_EPI_WARPS);
-        }
-        fence_barrier_init();
-    }
-    if (warp == 1) {
-        tcgen05_alloc(smem_u32(tmem_slot), TMEM_COLS);
-        tcgen05_relinquish();
-    }
-    tcgen05_fence_before();
-    __syncthreads();
-    tcgen05_fence_after();
-    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
-
-    bool ok = true;
-    TileWalk walk(p, (int)blockIdx.x, (int)gridDim.x, BN);
-    SubTile t;
-    if (warp == 0) {
-        // ---- stage 1: activation tiles and packed weight tiles by TMA -------------------------
-        if (lane == 0) {
-            uint32_t it = 0;
-            while (ok && walk.next(t)) {
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = (int)(it % NSTAGE);
-                    const uint32_t ph = (it / NSTAGE) & 1u;
-                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
-                    mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + P_STAGE_BYTES);
-                    tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, t.tile_m * (BM * MH), loaded0 + 8 * s);
-#pragma unroll
-                    for (int i = 0; i < BITS; ++i)
-                        tma_load_3d(smem_u32(p_tiles + s * P_STAGE_BYTES + i * P_PLANE_BYTES), &tmap_w, kb * (BK / 8), i,
-                                    t.col0 / 4, loaded0 + 8 * s);
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ---- stage 3: tensor-core MMA --------------------------------------------------------
-        if (lane == 0) {
-            uint32_t it = 0, ti = 0;
-            while (ok && walk.next(t)) {
-                const uint32_t buf = ti % NACC, aph = (ti / NACC) & 1u;
-                if (!mbar_wait(acce0 + 8 * buf, aph ^ 1u)) { ok = false; break; }
-                tcgen05_fence_after();
-                const uint32_t idesc = (1u << 4) | ((uint32_t)(t.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = (int)(it % NSTAGE);
-                    const uint32_t ph = (it / NSTAGE) & 1u;
-                    if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
-                    tcgen05_fence_after();
-                    const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
-#pragma unroll
-                    for (int j = 0; j < BK / 16; ++j)
-#pragma unroll
-                        for (int h = 0; h < MH; ++h) {
-                            const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES + h * A_HALF_BYTES));
-                            tcgen05_mma_f16(tmem_base + buf * ACC_COLS + (uint32_t)(h * BN), adesc + 2 * j, bdesc + 2 * j, idesc,
-                                            (kb > 0 || j > 0) ? 1u : 0u);
-                        }
-                    tcgen05_commit(empty0 + 8 * s);
-                }
-                if (ok) tcgen05_commit(accf0 + 8 * buf);
-                ++ti;
-            }
-        }
-    } else if (warp < 2 + NUM_DEQ_WARPS) {
-        // ---- stage 2: two-level lookup dequantization ----------------------------------------
-        // A warp owns 16 columns and both plane words of a k-block: lane = (strip of the warp, word,
-        // column of the strip).  With this split the 32 lanes read 32 different banks of the staged
-        // plane words and write eight different 16-byte bank groups per quarter-warp.
-        // Sub-tiles of at most 128 columns need only half of the warps per k-block: the two halves
-        // then take turns, two k-blocks each, so that all sixteen warps still share the work.
-        const int wd16 = warp - 2;
-        const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
-        const int nblk = p.K / p.group;
-        const int gshift = (p.group == 32) ? 5 : (p.group == 64) ? 6 : 7;
-        auto block_of = [&](int kb) { return ((2 * kb + v) * 32) >> gshift; };
-
-        uint32_t it0 = 0;                                  // pipeline position of the sub-tile's first k-block
-        while (ok && walk.next(t)) {
-            const int ngroups = (t.bn <= 128) ? 2 : 1;   // eight warps cover 128 columns
-            const int wd = (ngroups == 2) ? (wd16 & (NUM_DEQ_WARPS / 2 - 1)) : wd16;
-            const int grp = (ngroups == 2) ? wd16 / (NUM_DEQ_WARPS / 2) : 0;
-            const int n_local = wd * 16 + sl * 4 + c;
-            const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
-            const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
-            const uint32_t xr = (uint32_t)(n_local & 7);
-            const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
-            // k-blocks this warp works on: all of them, or every other pair (num_kb is even)
-            auto mine = [&](int kb) { return ngroups == 1 || ((kb >> 1) & 1) == grp; };
-            auto next_mine = [&](int kb) { return (ngroups == 1 || !(kb & 1)) ? kb + 1 : kb + 3; };
-            const int n = t.col0 + n_local;
-            const bool valid = n_local < t.bn && n < p.N;   // columns past the sub-tile are not used by the MMA
-            const int nb = n >> 2;
-            const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
-            const uint16_t *pz = p.zeros + (size_t)nb * nblk;
-            auto fetch_sz = [&](int B, __half &sv, uint32_t &zz) {
-                sv = __float2half(0.f);
-                zz = 0u;
-                if (valid && B < nblk) {
-                    sv = __ldg(ps + (size_t)B * 4);
-                    zz = ((uint32_t)__ldg(pz + B) >> (4 * c)) & 0xFu;
-                }
-            };
-            ConvTable<BITS> T;
-            int cur_B = -1, next_B = -1;
-            __half sv_next = __float2half(0.f);
-            uint32_t zz_next = 0u;
-
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const uint32_t it = it0 + (uint32_t)kb;
-                const int s = (int)(it % NSTAGE);
-                const uint32_t ph = (it / NSTAGE) & 1u;
-                const bool work = valid && mine(kb);
-                if (work) {
-                    const int Bk = block_of(kb);
-                    if (Bk != cur_B) {
-                        if (next_B != Bk) fetch_sz(Bk, sv_next, zz_next);
-                        cur_B = Bk;
-                        T.build(sv_next, zz_next);
-                    }
-                    // scale and zero-point of the block after this one are fetched one k-block ahead
-                    const int kn = next_mine(kb);
-                    const int Bn = block_of(kn);
-                    if (kn < num_kb && Bn != cur_B && Bn != next_B) {
-                        next_B = Bn;
-                        fetch_sz(Bn, sv_next, zz_next);
-                    }
-                }
-                if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
-                if (work) {
-                    uint32_t w[BITS];
-                    const uint32_t pp = p_base + (uint32_t)s * P_STAGE_BYTES;
-#pragma unroll
-                    for (int i = 0; i < BITS; ++i)
-                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[i]) : "r"(pp + i * P_PLANE_BYTES) : "memory");
-                    uint32_t out[16];
-                    dequant_word<BITS>(w, T, out);
-                    const uint32_t row = b_base + (uint32_t)s * B_STAGE_BYTES;
-#pragma unroll
-                    for (int cj = 0; cj < 4; ++cj) {
-                        const uint32_t chunk = ((uint32_t)(4 * v + cj)) ^ xr;
-                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(row + chunk * 16u), "r"(out[4 * cj]),
-                                     "r"(out[4 * cj + 1]), "r"(out[4 * cj + 2]), "r"(out[4 * cj + 3]) : "memory");
-                    }
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full0 + 8 * s);
-            }
-            it0 += (uint32_t)num_kb;
-        }
-    } else {
-        // ---- epilogue: tensor memory -> fp16 -> global, one warp per quarter of the lanes --------
-        const int quarter = warp & 3;                      // tensor-memory lanes this warp may read
-        const int epart = (warp - 2 - NUM_DEQ_WARPS) >> 2; // which of the quarter's warps
-        uint32_t ti = 0;
-        while (ok && walk.next(t)) {
-            const uint32_t buf = ti % NACC, aph = (ti / NACC) & 1u;
-            if (!mbar_wait(accf0 + 8 * buf, aph)) { ok = false; break; }
-            tcgen05_fence_after();
-#pragma unroll 1
-            for (int h = 0; h < MH; ++h) {
-                const int m = t.tile_m * (BM * MH) + h * BM + quarter * 32 + lane;
-#pragma unroll 1
-                for (int col = 32 * epart; col < t.bn; col += 32 * (NUM_EPI_WARPS / 4)) {
-                    uint32_t r[32];
-                    tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * ACC_COLS + (uint32_t)(h * BN + col), r);
-                    tcgen05_wait_ld();
-                    if (m < p.M) {
-                        __half *dst = p.y + (size_t)m * p.N + (size_t)t.col0 + col;
-#pragma unroll
-                        for (int g8 = 0; g8 < 4; ++g8) {
-                            if (col + 8 * g8 < t.bn && t.col0 + col + 8 * g8 < p.N) {
-                                uint32_t hv[4];
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const __half2 hh = __floats2half2_rn(__uint_as_float(r[8 * g8 + 2 * e]),
-                                                                         __uint_as_float(r[8 * g8 + 2 * e + 1]));
-                                    hv[e] = *reinterpret_cast<const uint32_t *>(&hh);
-                                }
-                                *reinterpret_cast<uint4 *>(dst + 8 * g8) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
-                            }
-                        }
-                    }
-                }
-            }
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acce0 + 8 * buf);
-            ++ti;
-        }
-    }
-
-    if (!ok) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
-    tcgen05_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tcgen05_fence_after();
-        tcgen05_dealloc(tmem_base, TMEM_COLS);
-    }
-}
-
-// ---- CTA-pair variant ------------------------------------------------------------------------
-// Two CTAs of a cluster share one tile of 2*128*MH tokens x up to 256 output channels: each holds its
-// own 128*MH token rows, dequantizes half of the tile's channels, and the pair multiplies with
-// tcgen05.mma.cta_group::2 (M = 256), issued by the pair's first CTA.  Each SM then reads only half of
-// the weight tile per MMA and dequantizes half as much per flop, which is what the single-CTA kernel
-// is short of (shared-memory bandwidth, ALU pipe).  Barriers that both CTAs feed (weight tile ready,
-// accumulator drained) live in the first CTA and are reached with cluster-scope arrives; the MMA's
-// commits arrive in both CTAs.  No TMA multicast is used: each CTA loads its own tiles.
-constexpr int PAIR_BN = 256;                     // channels of a pair tile (128 per CTA)
-constexpr int PAIR_NSTAGE = 4;
-constexpr int PAIR_B_STAGE_BYTES = (PAIR_BN / 2) * BK * 2;
-constexpr int PAIR_P_PLANE_BYTES = (PAIR_BN / 8) * (BK / 32) * 16;
-constexpr int PAIR_OUT_BYTES = 32 * 32 * 2;      // an epilogue warp's output staging: 32 tokens x 32 channels
-constexpr int pair_smem_bytes(int mh, int bits)
-{
-    // stages, barriers (256 B), staging (1024-aligned as the stages are: bits * 1 KB keeps it so), slack to align
-    return PAIR_NSTAGE * (mh * A_HALF_BYTES + PAIR_B_STAGE_BYTES + bits * PAIR_P_PLANE_BYTES) + 1024
-           + NUM_EPI_WARPS * PAIR_OUT_BYTES + 256;
-}
-
-template <int BITS, int MH>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
-mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                   const __grid_constant__ CUtensorMap tmap_y, const GemmParams p)
-{
-    constexpr int NSTAGE = PAIR_NSTAGE, B_STAGE_BYTES = PAIR_B_STAGE_BYTES, P_PLANE_BYTES = PAIR_P_PLANE_BYTES;
-    constexpr int A_STAGE_BYTES = MH * A_HALF_BYTES;
-    constexpr int P_STAGE_BYTES = BITS * P_PLANE_BYTES;
-    constexpr int TMEM_COLS = MH * PAIR_BN;            // MH accumulators of 256 columns (512 for MH = 2)
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t rank = cluster_ctarank();           // 0: issues the MMAs and owns the shared barriers
-    const bool hdr_ok = header_matches(p.packed, p.K, p.N, p.bits, p.group);   // same answer in every CTA
-    if (!hdr_ok) {
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // in a pair, CTA 0 issues the MMAs and owns the shared barriers
+    if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {   // same answer in every CTA
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
         return;
     }
@@ -665,53 +456,75 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     uint8_t *b_tiles = smem + NSTAGE * A_STAGE_BYTES;
     uint8_t *p_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES);
     uint8_t *out_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + P_STAGE_BYTES);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(out_tiles + NUM_EPI_WARPS * PAIR_OUT_BYTES);
-    // bars[0..NSTAGE) loaded (own TMA), [NSTAGE..2NSTAGE) full (both CTAs' dequantization warps; used in
-    // CTA 0), [2NSTAGE..3NSTAGE) empty (MMA commit, both CTAs), then accumulator full (commit, both CTAs)
-    // and accumulator empty (both CTAs' epilogue warps; used in CTA 0)
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * NSTAGE + 2);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(out_tiles + NUM_EPI_WARPS * OUT_TILE_BYTES);
+    // bars[0..NSTAGE) loaded (own TMA), [NSTAGE..2NSTAGE) full (dequantized; in a pair both CTAs' warps
+    // arrive in CTA 0), [2NSTAGE..3NSTAGE) empty (MMA commit), then accumulator full (commit) and
+    // accumulator empty (epilogue warps; in a pair both CTAs' warps arrive in CTA 0)
+    // and PART_RING barriers per epilogue warp for the partial chunks it fetches
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * NSTAGE + 2 + NUM_EPI_WARPS * PART_RING);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = p.K / BK;
     const uint32_t loaded0 = smem_u32(bars), full0 = smem_u32(bars + NSTAGE), empty0 = smem_u32(bars + 2 * NSTAGE),
-                   accf = smem_u32(bars + 3 * NSTAGE), acce = smem_u32(bars + 3 * NSTAGE + 1);
+                   accf = smem_u32(bars + 3 * NSTAGE), acce = smem_u32(bars + 3 * NSTAGE + 1),
+                   ring0 = smem_u32(bars + 3 * NSTAGE + 2);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(loaded0 + 8 * s, 1);
-            mbar_init(full0 + 8 * s, 2 * NUM_DEQ_WARPS);
+            mbar_init(full0 + 8 * s, NCTA * NUM_DEQ_WARPS);
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accf, 1);
-        mbar_init(acce, 2 * NUM_EPI_WARPS);
+        mbar_init(acce, NCTA * NUM_EPI_WARPS);
+        for (int b = 0; b < NUM_EPI_WARPS * PART_RING; ++b) mbar_init(ring0 + 8 * b, 1);
         *tmem_slot = 0xFFFFFFFFu;
         fence_barrier_init();
     }
     __syncthreads();
     if (warp == 1) {
-        tcgen05_alloc2(smem_u32(tmem_slot), TMEM_COLS);
-        tcgen05_relinquish2();
+        if constexpr (PAIR) {
+            tcgen05_alloc2(smem_u32(tmem_slot), TMEM_COLS);
+            tcgen05_relinquish2();
+        } else {
+            tcgen05_alloc(smem_u32(tmem_slot), TMEM_COLS);
+            tcgen05_relinquish();
+        }
     }
     tcgen05_fence_before();
     __syncthreads();
-    cluster_sync_all();                                // both CTAs' barriers and tensor memory are set up
+    if constexpr (PAIR) cluster_sync_all();            // both CTAs' barriers and tensor memory are set up
     tcgen05_fence_after();
     uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
-    if (tmem_base == 0xFFFFFFFFu) tmem_base = ld_shared_cluster_u32(mapa_u32(smem_u32(tmem_slot), rank ^ 1u));
+    if constexpr (PAIR)
+        if (tmem_base == 0xFFFFFFFFu) tmem_base = ld_shared_cluster_u32(mapa_u32(smem_u32(tmem_slot), rank ^ 1u));
 
     bool ok = tmem_base != 0xFFFFFFFFu;
-    // the pair walks through its items together; a CTA's rows and channels inside a sub-tile:
-    TileWalk walk(p, (int)(blockIdx.x >> 1), (int)(gridDim.x >> 1), PAIR_BN, 32);
-    SubTile t;
-    const uint32_t full_lead = mapa_u32(full0, 0), acce_lead = mapa_u32(acce, 0);
+    const int worker = (int)blockIdx.x / NCTA, nworkers = (int)gridDim.x / NCTA;
+    Span span(p, worker, nworkers);
+    Segment sg;
+    // a tile's place in the output, the channels this CTA dequantizes (a pair halves the tile's channels;
+    // the last tile of a row may be narrower: a multiple of 32 channels that reaches N)
+    auto tile_rows = [&](int tile) { return (tile % p.tiles_m) * (NCTA * ROWS_CTA) + (int)rank * ROWS_CTA; };
+    // (the N/32 column units are cut into tiles_n column tiles of almost equal width, at most BN)
+    const int n32 = (p.N + 31) / 32;
+    auto tile_unit0 = [&](int ct) { return (int)(((long long)n32 * ct) / p.tiles_n); };
+    auto tile_col0 = [&](int tile) { return 32 * tile_unit0(tile / p.tiles_m); };
+    auto tile_bn = [&](int tile) { const int ct = tile / p.tiles_m; return 32 * (tile_unit0(ct + 1) - tile_unit0(ct)); };
+    const uint32_t full_lead = PAIR ? mapa_u32(full0, 0) : full0, acce_lead = PAIR ? mapa_u32(acce, 0) : acce;
+    auto arrive_lead = [&](uint32_t bar) {
+        if constexpr (PAIR) mbar_arrive_cluster(bar);
+        else mbar_arrive(bar);
+    };
+
     if (warp == 0) {
         // ---- stage 1: this CTA's activation rows and packed channels by TMA ---------------------
         if (lane == 0) {
             uint32_t it = 0;
-            while (ok && walk.next(t)) {
-                const int row0 = t.tile_m * (2 * BM * MH) + (int)rank * (BM * MH);
-                const int strip0 = (t.col0 + (int)rank * (t.bn / 2)) / 4;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            while (ok && span.next(sg)) {
+                const int row0 = tile_rows(sg.tile);
+                const int strip0 = (tile_col0(sg.tile) + (int)rank * (tile_bn(sg.tile) / NCTA)) / 4;
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
                     const int s = (int)(it % NSTAGE);
                     const uint32_t ph = (it / NSTAGE) & 1u;
                     if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
@@ -725,14 +538,14 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             }
         }
     } else if (warp == 1) {
-        // ---- stage 3: the pair's MMAs, issued by CTA 0 ------------------------------------------
+        // ---- stage 3: tensor-core MMA (in a pair: issued by CTA 0 for both) ----------------------
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, ti = 0;
-            while (ok && walk.next(t)) {
+            while (ok && span.next(sg)) {
                 if (!mbar_wait(acce, (ti & 1u) ^ 1u)) { ok = false; break; }
                 tcgen05_fence_after();
-                const uint32_t idesc = (1u << 4) | ((uint32_t)(t.bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const uint32_t idesc = (1u << 4) | ((uint32_t)(tile_bn(sg.tile) >> 3) << 17) | ((uint32_t)((NCTA * BM) >> 4) << 24);
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
                     const int s = (int)(it % NSTAGE);
                     const uint32_t ph = (it / NSTAGE) & 1u;
                     if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
@@ -743,20 +556,28 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
 #pragma unroll
                         for (int h = 0; h < MH; ++h) {
                             const uint64_t adesc = make_kmajor_sw128_desc(smem_u32(a_tiles + s * A_STAGE_BYTES + h * A_HALF_BYTES));
-                            tcgen05_mma2_f16(tmem_base + (uint32_t)(h * PAIR_BN), adesc + 2 * j, bdesc + 2 * j, idesc,
-                                             (kb > 0 || j > 0) ? 1u : 0u);
+                            const uint32_t acc = (kb > sg.kb0 || j > 0) ? 1u : 0u;
+                            if constexpr (PAIR) tcgen05_mma2_f16(tmem_base + (uint32_t)(h * BN), adesc + 2 * j, bdesc + 2 * j, idesc, acc);
+                            else tcgen05_mma_f16(tmem_base + (uint32_t)(h * BN), adesc + 2 * j, bdesc + 2 * j, idesc, acc);
                         }
-                    tcgen05_commit2_both(empty0 + 8 * s);
+                    if constexpr (PAIR) tcgen05_commit2_both(empty0 + 8 * s);
+                    else tcgen05_commit(empty0 + 8 * s);
                 }
-                if (ok) tcgen05_commit2_both(accf);
+                if (ok) {
+                    if constexpr (PAIR) tcgen05_commit2_both(accf);
+                    else tcgen05_commit(accf);
+                }
                 ++ti;
             }
         }
     } else if (warp < 2 + NUM_DEQ_WARPS) {
-        // ---- stage 2: two-level lookup dequantization of this CTA's half of the channels --------
-        // at most 128 channels per CTA: the two halves of the sixteen warps take turns, two k-blocks each
+        // ---- stage 2: two-level lookup dequantization of this CTA's channels ----------------------
+        // A warp owns 16 channels and both plane words of a k-block: lane = (strip of the warp, word,
+        // column of the strip).  With this split the 32 lanes read 32 different banks of the staged
+        // plane words and write eight different 16-byte bank groups per quarter-warp.  A CTA of a pair
+        // has 128 channels: the two halves of its sixteen warps take turns, two k-blocks each.
         const int wd16 = warp - 2;
-        const int wd = wd16 & (NUM_DEQ_WARPS / 2 - 1), grp = wd16 / (NUM_DEQ_WARPS / 2);
+        const int wd = wd16 % (NUM_DEQ_WARPS / NGROUP), grp = wd16 / (NUM_DEQ_WARPS / NGROUP);
         const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
         const int nblk = p.K / p.group;
         const int gshift = (p.group == 32) ? 5 : (p.group == 64) ? 6 : 7;
@@ -766,14 +587,14 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
         const uint32_t xr = (uint32_t)(n_local & 7);
         const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
-        auto mine = [&](int kb) { return ((kb >> 1) & 1) == grp; };
-        auto next_mine = [&](int kb) { return !(kb & 1) ? kb + 1 : kb + 3; };
+        // k-blocks this warp works on, by pipeline position (segments start at even k-blocks)
+        auto mine = [&](uint32_t it) { return NGROUP == 1 || (int)((it >> 1) & 1u) == grp; };
 
-        uint32_t it0 = 0;
-        while (ok && walk.next(t)) {
-            const int half = t.bn / 2;
-            const int n = t.col0 + (int)rank * half + n_local;
-            const bool valid = n_local < half && n < p.N;
+        uint32_t it = 0;
+        while (ok && span.next(sg)) {
+            const int chans = tile_bn(sg.tile) / NCTA;
+            const int n = tile_col0(sg.tile) + (int)rank * chans + n_local;
+            const bool valid = n_local < chans && n < p.N;   // channels past the tile are not used by the MMA
             const int nb = n >> 2;
             const __half *ps = p.scales + (size_t)nb * nblk * 4 + c;
             const uint16_t *pz = p.zeros + (size_t)nb * nblk;
@@ -789,11 +610,10 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             int cur_B = -1, next_B = -1;
             __half sv_next = __float2half(0.f);
             uint32_t zz_next = 0u;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const uint32_t it = it0 + (uint32_t)kb;
+            for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
                 const int s = (int)(it % NSTAGE);
                 const uint32_t ph = (it / NSTAGE) & 1u;
-                const bool work = valid && mine(kb);
+                const bool work = valid && mine(it);
                 if (work) {
                     const int Bk = block_of(kb);
                     if (Bk != cur_B) {
@@ -801,9 +621,10 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         cur_B = Bk;
                         T.build(sv_next, zz_next);
                     }
-                    const int kn = next_mine(kb);
+                    // scale and zero-point of the block after this one are fetched one k-block ahead
+                    const int kn = (NGROUP == 1 || !(kb & 1)) ? kb + 1 : kb + 3;
                     const int Bn = block_of(kn);
-                    if (kn < num_kb && Bn != cur_B && Bn != next_B) {
+                    if (kn < sg.kb1 && Bn != cur_B && Bn != next_B) {
                         next_B = Bn;
                         fetch_sz(Bn, sv_next, zz_next);
                     }
@@ -827,64 +648,151 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(full_lead + 8 * s);
+                if (lane == 0) arrive_lead(full_lead + 8 * s);
             }
-            it0 += (uint32_t)num_kb;
         }
     } else {
-        // ---- epilogue: this CTA's rows, tensor memory -> fp16 -> shared memory -> global (tile stores) --
-        // A warp reads 32 tokens x 32 channels (one token per lane), writes them as 64-byte rows into its
-        // staging tile in the 64-byte swizzle (16-byte chunk index ^ bits 1..2 of the row: no bank
-        // conflicts) and one lane stores the tile; tokens >= M and channels >= N are clipped by the store.
+        // ---- epilogue: this CTA's rows of a segment's accumulators ------------------------------------
+        // A warp reads chunks of 32 tokens x 32 channels (one token per lane; a warp may only read its
+        // quarter of the tensor-memory lanes).  Whole tiles and the finishing segment of a split tile:
+        // round to fp16, write 64-byte rows into the warp's staging tile in the 64-byte swizzle (16-byte
+        // chunk index ^ bits 1..2 of the row: no bank conflicts), one lane stores the tile (tokens >= M
+        // and channels >= N are clipped by the store).  Split tiles: the other segments write the fp32
+        // chunks to this CTA's partial tile and raise the warp's flag.  The finishing segment, always
+        // the last of its worker's walk, waits for the flags of the same warp in the workers before it,
+        // fetches their chunks with bulk copies into the pipeline's stage buffers (free by then; a ring
+        // of PART_RING chunks per warp keeps enough bytes in flight) and adds them in worker order.
         const int quarter = warp & 3;
         const int ew = warp - 2 - NUM_DEQ_WARPS, epart = ew >> 2;
-        const uint32_t stage = smem_u32(out_tiles + ew * PAIR_OUT_BYTES);
+        const uint32_t stage = smem_u32(out_tiles + ew * OUT_TILE_BYTES);
         const uint32_t my_row = stage + (uint32_t)lane * 64u, xr = ((uint32_t)lane >> 1) & 3u;
+        const uint32_t ring_buf = smem_u32(smem) + (uint32_t)ew * (PART_RING * CHUNK_BYTES);
+        const uint32_t ring_bar = ring0 + 8u * (uint32_t)(ew * PART_RING);
+        constexpr size_t WARP_PARTIAL_FLOATS = (size_t)MH * (BN / 64) * (CHUNK_BYTES / 4);
+        static_assert(NUM_EPI_WARPS * PART_RING * CHUNK_BYTES <= NSTAGE * A_STAGE_BYTES + NSTAGE * B_STAGE_BYTES, "ring fits in the stages");
+        auto warp_partial = [&](int cta) { return p.partial + ((size_t)cta * NUM_EPI_WARPS + ew) * WARP_PARTIAL_FLOATS; };
+        auto warp_flag = [&](int cta) { return p.flags + (size_t)cta * NUM_EPI_WARPS + ew; };
         uint32_t ti = 0;
-        while (ok && walk.next(t)) {
+        while (ok && span.next(sg)) {
+            const int bn = tile_bn(sg.tile), col0 = tile_col0(sg.tile), rows0 = tile_rows(sg.tile);
+            // this warp's chunks: nch column chunks for each of the hv row blocks that reach below M
+            const int nch = (bn - 32 * epart + 63) / 64;
+            int hv = 0;
+            for (int h = 0; h < MH; ++h) hv += (rows0 + h * BM + quarter * 32 < p.M) ? 1 : 0;
+            const int nq = hv * nch;
+            // split tile: the workers before this one that hold the tile's other segments
+            int first_w = worker;
+            if (sg.finishes && !sg.whole) first_w = span.owner(sg.tile, 0);
+            const int ncontrib = worker - first_w;
             if (!mbar_wait(accf, ti & 1u)) { ok = false; break; }
             tcgen05_fence_after();
-            bool released = false;
-#pragma unroll 1
-            for (int h = 0; h < MH; ++h) {
-                const int m0 = t.tile_m * (2 * BM * MH) + (int)rank * (BM * MH) + h * BM + quarter * 32;
-#pragma unroll 1
-                for (int col = 32 * epart; col < t.bn; col += 32 * (NUM_EPI_WARPS / 4)) {
-                    const bool last = (h == MH - 1) && (col + 32 * (NUM_EPI_WARPS / 4) >= t.bn);
-                    uint32_t r[32];
-                    if (m0 < p.M) {
-                        tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * PAIR_BN + col), r);
-                        tcgen05_wait_ld();
-                    }
-                    if (last) {                        // the accumulators are read: the next tile's MMAs may start
-                        tcgen05_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_cluster(acce_lead);
-                        released = true;
-                    }
-                    if (m0 < p.M) {
-                        uint32_t hv[16];
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const __half2 hh = __floats2half2_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                            hv[e] = *reinterpret_cast<const uint32_t *>(&hh);
+            // issue the fetch of item j = (chunk q, contributor c) into the ring (lane 0)
+            auto fetch = [&](int j) {
+                const int q = j / ncontrib, cw = first_w + j % ncontrib;
+                const size_t off = (size_t)((q / nch) * (BN / 64) + (q % nch)) * (CHUNK_BYTES / 4);
+                const uint32_t b = (uint32_t)(j % PART_RING);
+                mbar_expect_tx(ring_bar + 8 * b, CHUNK_BYTES);
+                bulk_load(ring_buf + b * CHUNK_BYTES, warp_partial(cw * NCTA + (int)rank) + off, CHUNK_BYTES, ring_bar + 8 * b);
+            };
+            if (ncontrib > 0) {
+                // their partial tiles were written at the start of their walks; bounded wait all the same
+                if (lane == 0) {
+                    for (int cw = first_w; cw < worker && ok; ++cw) {
+                        const uint32_t *f = warp_flag(cw * NCTA + (int)rank);
+                        uint64_t t0 = 0;
+                        for (uint32_t spin = 0;; ++spin) {
+                            uint32_t fv;
+                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(fv) : "l"(f) : "memory");
+                            if (fv == 1u) break;
+                            if ((spin & 255u) == 255u) {
+                                const uint64_t now = global_timer_ns();
+                                if (t0 == 0) t0 = now;
+                                else if (now - t0 > 1000000000ull) { ok = false; break; }
+                            }
                         }
-                        if (lane == 0) tma_store_wait_read();      // the staging tile is free again
-                        __syncwarp();
-#pragma unroll
-                        for (uint32_t cj = 0; cj < 4; ++cj)
-                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((cj ^ xr) << 4)), "r"(hv[4 * cj]),
-                                         "r"(hv[4 * cj + 1]), "r"(hv[4 * cj + 2]), "r"(hv[4 * cj + 3]) : "memory");
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) tma_store_2d(&tmap_y, stage, t.col0 + col, m0);
+                    }
+                    if (ok) {
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                        for (int j = 0; j < PART_RING && j < nq * ncontrib; ++j) fetch(j);
                     }
                 }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
             }
-            if (!released) {                           // a warp without a chunk in this sub-tile
+            float *mine_partial = warp_partial((int)blockIdx.x);
+            if (nq == 0) {                             // a warp without a chunk in this tile
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(acce_lead);
+                if (lane == 0) arrive_lead(acce_lead);
+            }
+            int j = 0;                                 // next item of the ring to consume
+#pragma unroll 1
+            for (int q = 0; q < nq; ++q) {
+                const int h = q / nch, col = 32 * epart + 64 * (q % nch);
+                const int m0 = rows0 + h * BM + quarter * 32;
+                uint32_t r[32];
+                tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * BN + col), r);
+                tcgen05_wait_ld();
+                if (q == nq - 1) {                     // the accumulators are read: the next segment's MMAs may start
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) arrive_lead(acce_lead);
+                }
+                if (!sg.finishes) {
+                    // chunk as eight rows of 32 float4: coalesced, and fetched back as one 4 KB block
+                    float4 *dst = reinterpret_cast<float4 *>(mine_partial + (size_t)(h * (BN / 64) + (q % nch)) * (CHUNK_BYTES / 4)) + lane;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        __stcg(dst + 32 * e, make_float4(__uint_as_float(r[4 * e]), __uint_as_float(r[4 * e + 1]),
+                                                         __uint_as_float(r[4 * e + 2]), __uint_as_float(r[4 * e + 3])));
+                    continue;
+                }
+#pragma unroll 1
+                for (int c = 0; c < ncontrib; ++c, ++j) {
+                    const uint32_t b = (uint32_t)(j % PART_RING);
+                    if (!mbar_wait(ring_bar + 8 * b, (uint32_t)(j / PART_RING) & 1u)) { ok = false; break; }
+                    const uint32_t src = ring_buf + b * CHUNK_BYTES + (uint32_t)lane * 16u;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        float4 a;
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w)
+                                     : "r"(src + 512u * e) : "memory");
+                        r[4 * e]     = __float_as_uint(__uint_as_float(r[4 * e]) + a.x);
+                        r[4 * e + 1] = __float_as_uint(__uint_as_float(r[4 * e + 1]) + a.y);
+                        r[4 * e + 2] = __float_as_uint(__uint_as_float(r[4 * e + 2]) + a.z);
+                        r[4 * e + 3] = __float_as_uint(__uint_as_float(r[4 * e + 3]) + a.w);
+                    }
+                    __syncwarp();                      // every lane has read the buffer: it may be refilled
+                    if (lane == 0 && j + PART_RING < nq * ncontrib) fetch(j + PART_RING);
+                }
+                if (!ok) break;
+                uint32_t hv16[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const __half2 hh = __floats2half2_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                    hv16[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                }
+                if (lane == 0) tma_store_wait_read();              // the staging tile is free again
+                __syncwarp();
+#pragma unroll
+                for (uint32_t cj = 0; cj < 4; ++cj)
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((cj ^ xr) << 4)), "r"(hv16[4 * cj]),
+                                 "r"(hv16[4 * cj + 1]), "r"(hv16[4 * cj + 2]), "r"(hv16[4 * cj + 3]) : "memory");
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) tma_store_2d(&tmap_y, stage, col0 + col, m0);
+            }
+            if (!ok) break;
+            if (!sg.finishes) {
+                // partial tile complete: every lane's stores, then the flag
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(warp_flag((int)blockIdx.x)), "r"(1u) : "memory");
+            } else if (ncontrib > 0) {
+                // the partial tiles are consumed: their flags go back to "empty" for the next launch
+                __syncwarp();
+                if (lane == 0)
+                    for (int cw = first_w; cw < worker; ++cw) *warp_flag(cw * NCTA + (int)rank) = kFlagEmpty;
             }
             ++ti;
         }
@@ -894,10 +802,11 @@ mpgemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     if (!ok) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
     tcgen05_fence_before();
     __syncthreads();
-    cluster_sync_all();                                // nobody touches the peer's memory after this
+    if constexpr (PAIR) cluster_sync_all();            // nobody touches the peer's memory after this
     if (warp == 1 && tmem_base != 0xFFFFFFFFu) {
         tcgen05_fence_after();
-        tcgen05_dealloc2(tmem_base, TMEM_COLS);
+        if constexpr (PAIR) tcgen05_dealloc2(tmem_base, TMEM_COLS);
+        else tcgen05_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -916,56 +825,91 @@ EncodeTiledFn encode_fn()
     return reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-template <int BITS, int MH, int WIDE>
-tman_status launch_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const GemmParams &p, cudaStream_t s)
-{
-    auto kern = mpgemm_kernel<BITS, MH, WIDE>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<WIDE>(MH, BITS)) != cudaSuccess)
-        return TMAN_ERR_CUDA;
-    // one CTA per SM (fewer when there are fewer items than that): every CTA walks through its items
-    long long grid = p.sms;
-    if (grid > (long long)p.tiles_m * p.R) grid = (long long)p.tiles_m * p.R;
-    kern<<<(unsigned)grid, GEMM_THREADS, smem_bytes<WIDE>(MH, BITS), s>>>(tmap_x, tmap_w, p);
-    return launch_status();
-}
+// Row blocks per CTA and single CTAs or pairs, from the number of tokens: one CTA up to 128 tokens,
+// pairs of one row block each up to 256, pairs of two row blocks each beyond.
+inline int gemm_mh(int M) { return M > 2 * BM ? 2 : 1; }
+inline bool gemm_pair(int M) { return M > BM; }
 
-template <int BITS, int MH>
-tman_status launch_pair_tile(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y,
-                             const GemmParams &p, cudaStream_t s)
+template <int BITS, int MH, bool PAIR>
+tman_status launch_cfg(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const GemmParams &p,
+                       int sms, cudaStream_t s)
 {
-    auto kern = mpgemm_pair_kernel<BITS, MH>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pair_smem_bytes(MH, BITS)) != cudaSuccess)
+    using C = Cfg<MH, PAIR>;
+    auto kern = mpgemm_kernel<BITS, MH, PAIR>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes(BITS)) != cudaSuccess)
         return TMAN_ERR_CUDA;
-    long long pairs = p.sms / 2;
-    if (pairs > (long long)p.tiles_m * p.R) pairs = (long long)p.tiles_m * p.R;
+    // One worker per SM (pair of SMs), fewer when there is less work than that.  The channels are cut
+    // into column tiles of almost equal width (multiples of 32, at most 256) and the tiles dealt whole;
+    // the number of column tiles is the one with the least estimated time for the longest worker:
+    // rounds of tiles x k-blocks x time of a k-block, which for a pair hardly falls below 192 channels
+    // (the MMA's activation operand bounds it) and for a single CTA is the dequantization's, in
+    // proportion to the width (measured figures, microseconds).  The alternative: the widest tiles,
+    // whole as far as they go round and the rest in equal spans, whose split tiles cost their workers a
+    // partial tile written to and read back from the workspace (an SM writes about 50 GB/s).
+    const long long nu = p.K / (2 * BK);
+    long long workers = (sms < kMaxGemmCtas ? sms : kMaxGemmCtas) / C::NCTA;
+    if (workers < 1) return TMAN_ERR_CUDA;
+    GemmParams q = p;
+    const int n32 = (p.N + 31) / 32, tn_min = (n32 + BN / 32 - 1) / (BN / 32);
+    auto kb_us = [](int width) {
+        const double w = (double)width;
+        return PAIR ? (0.0034 * w > 0.74 ? 0.0034 * w : 0.74) : (1.1 * w / 256 > 0.3 ? 1.1 * w / 256 : 0.3);
+    };
+    double best = 1e300;
+    q.whole_tiles = 1;
+    q.tiles_n = tn_min;
+    for (int tn = tn_min; tn <= n32 && tn <= 8 * tn_min; ++tn) {
+        const long long rounds = ((long long)p.tiles_m * tn + workers - 1) / workers;
+        const int wmax = 32 * ((n32 + tn - 1) / tn);
+        const double cost = (double)rounds * (2.0 * nu * kb_us(wmax) + 3.0);
+        if (cost < best - 1e-9) { best = cost; q.tiles_n = tn; }
+    }
+    {
+        const long long t = (long long)p.tiles_m * tn_min, rest = t % workers;
+        const double cost = (double)(t / workers) * (2.0 * nu * kb_us(BN) + 3.0) +
+                            (double)((rest * nu + workers - 1) / workers) * 2.0 * kb_us(BN) +
+                            (rest ? (PAIR ? 24.0 : 16.0) + 3.0 * (double)workers / (double)rest : 0.0);   // more pieces per tile: more to read back
+        if (rest != 0 && cost < best) {
+            q.whole_tiles = 0;
+            q.tiles_n = tn_min;
+        }
+    }
+    const long long tiles = (long long)q.tiles_m * q.tiles_n;
+    if (tiles < workers) {                             // fewer tiles than workers: as many workers as units at most
+        const long long units = q.whole_tiles ? tiles : tiles * nu;
+        if (workers > units) workers = units;
+    }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    cfg.gridDim = dim3((unsigned)(workers * C::NCTA));
     cfg.blockDim = dim3(GEMM_THREADS);
-    cfg.dynamicSmemBytes = pair_smem_bytes(MH, BITS);
+    cfg.dynamicSmemBytes = C::smem_bytes(BITS);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.x = C::NCTA;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, p) != cudaSuccess) return TMAN_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, q) != cudaSuccess) return TMAN_ERR_CUDA;
     return TMAN_OK;
 }
 
 template <int BITS>
-tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y,
-                        const GemmParams &p, int mh, cudaStream_t s)
+tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const GemmParams &p,
+                        int sms, cudaStream_t s)
 {
-    if (p.pair) return launch_pair_tile<BITS, 2>(tmap_x, tmap_w, tmap_y, p, s);   // pairs run on more than 256 tokens
-    if (p.wide) return mh == 2 ? launch_tile<BITS, 2, 1>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 1>(tmap_x, tmap_w, p, s);
-    return mh == 2 ? launch_tile<BITS, 2, 0>(tmap_x, tmap_w, p, s) : launch_tile<BITS, 1, 0>(tmap_x, tmap_w, p, s);
+    if (!gemm_pair(p.M)) return launch_cfg<BITS, 1, false>(tmap_x, tmap_w, tmap_y, p, sms, s);
+    if (gemm_mh(p.M) == 1) return launch_cfg<BITS, 1, true>(tmap_x, tmap_w, tmap_y, p, sms, s);
+    return launch_cfg<BITS, 2, true>(tmap_x, tmap_w, tmap_y, p, sms, s);
 }
 
 }  // namespace
 
-size_t mpgemm_workspace_bytes(int, int, int) { return kWsStatusBytes; }
+size_t mpgemm_workspace_bytes(int M, int, int)
+{
+    return kGemmPartialOff + (size_t)kMaxGemmCtas * partial_bytes_per_cta(gemm_mh(M));
+}
 
 tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t, cudaStream_t s)
@@ -973,88 +917,40 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     if ((reinterpret_cast<uintptr_t>(x) & 15) != 0 || (reinterpret_cast<uintptr_t>(y) & 15) != 0) return TMAN_ERR_SHAPE;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TMAN_ERR_CUDA;
-    CUtensorMap tmap;
-    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    // CTA pairs (each CTA 256 token rows of a 512-row tile, half of the tile's channels) when there
-    // are enough tokens and a pair of SMs gets a share of the output at least 192 channels wide;
-    // otherwise single CTAs, which waste less on narrow shares.
-    const int sms_q = sm_count();
-    if (sms_q <= 0) return TMAN_ERR_CUDA;
-    const long long share = (long long)N * ((M + 4 * BM - 1) / (4 * BM)) / (sms_q / 2 > 0 ? sms_q / 2 : 1);
-    const bool pair = M > 2 * BM && share >= 192;
-    const int mh = (M > BM) ? 2 : 1;                   // row blocks per CTA
-    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)(BM * mh)};
-    const cuuint32_t estr[2] = {1, 1};
-    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(x), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return TMAN_ERR_CUDA;
+    const int sms = sm_count();
+    if (sms <= 0) return TMAN_ERR_CUDA;
+    const int mh = gemm_mh(M);
+    const bool pair = gemm_pair(M);
+    const int rows_cta = BM * mh, bn_cta = pair ? BN / 2 : BN;
+    const cuuint32_t estr[3] = {1, 1, 1};
 
+    // activations: boxes of one k-block x a CTA's token rows, 128-byte swizzle
+    CUtensorMap tmap_x;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+        const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)rows_cta};
+        if (enc(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(x), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TMAN_ERR_CUDA;
+    }
     Layout L = make_layout(K, N, bits, group);
     const uint8_t *pk = static_cast<const uint8_t *>(packed);
-    GemmParams p;
-    p.packed = pk;
-    p.planes = reinterpret_cast<const uint32_t *>(pk + L.planes_off);
-    p.scales = reinterpret_cast<const __half *>(pk + L.scales_off);
-    p.zeros = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
-    p.y = static_cast<__half *>(y);
-    p.status = static_cast<uint32_t *>(ws);
-    p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
-    p.pair = pair ? 1 : 0;
-    p.tiles_m = pair ? (M + 2 * BM * mh - 1) / (2 * BM * mh) : (M + BM * mh - 1) / (BM * mh);
-    p.sms = sm_count();
-    if (p.sms <= 0) return TMAN_ERR_CUDA;
-    // Tile configuration and column ranges per row tile: the pair that minimises (waves of items over
-    // the SMs) x (cost of an item).  A sub-tile of w 16-column units costs about w + 10 units of
-    // shared-memory traffic per k-block (the activation tile is written once and read once per MMA
-    // whatever the width), and a wide sub-tile holds twice as many units as a narrow one.
-    if (pair) {
-        // pairs: units of 32 columns, sub-tiles of up to 8 units, one item at a time per pair of SMs
-        const int n32 = (N + 31) / 32, npairs = p.sms / 2;
-        double best = 1e300;
-        p.R = 1;
-        p.wide = 0;
-        for (int R = 1; R <= n32 && R <= 4096; ++R) {
-            const long long items = (long long)p.tiles_m * R;
-            const long long waves = (items + npairs - 1) / npairs;
-            const int w = (n32 + R - 1) / R;
-            const int nsub = (w + 7) / 8;
-            const double cost = (double)waves * (w + 3.0 * nsub);
-            if (cost < best - 1e-9) { best = cost; p.R = R; }
-        }
-    } else {
-        const int n16 = (N + 15) / 16;
-        double best = 1e300;
-        p.R = 1;
-        p.wide = 0;
-        for (int wide = 0; wide < 2; ++wide) {
-            const int maxw = (wide ? Cfg<1>::BN : Cfg<0>::BN) / 16;
-            for (int R = 1; R <= n16 && R <= 4096; ++R) {
-                const long long items = (long long)p.tiles_m * R;
-                const long long waves = (items + p.sms - 1) / p.sms;
-                const int w16 = (n16 + R - 1) / R;
-                const int nsub = (w16 + maxw - 1) / maxw;
-                const double cost = (double)waves * (w16 + 10.0 * nsub);
-                if (cost < best - 1e-9) { best = cost; p.R = R; p.wide = wide; }
-            }
-        }
-    }
     // the bit-plane words as a 3-D array of 32-bit elements: (word and column inside a strip's plane
-    // row, plane, strip); one box = the two words of a k-block for the strips of a tile, one plane
+    // row, plane, strip); one box = the two words of a k-block for the strips of a CTA's channels, one plane
     CUtensorMap tmap_w;
     {
         const cuuint64_t wt = (cuuint64_t)(K / 32);
         const cuuint64_t wdims[3] = {wt * 4, (cuuint64_t)bits, (cuuint64_t)(N / 4)};
         const cuuint64_t wstrides[2] = {wt * 16, wt * 16 * (cuuint64_t)bits};
-        const cuuint32_t wbox[3] = {(cuuint32_t)(BK / 8), 1, (cuuint32_t)((pair ? PAIR_BN / 2 : (p.wide ? Cfg<1>::BN : Cfg<0>::BN)) / 4)};
-        const cuuint32_t westr[3] = {1, 1, 1};
+        const cuuint32_t wbox[3] = {(cuuint32_t)(BK / 8), 1, (cuuint32_t)(bn_cta / 4)};
         if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t *>(pk + L.planes_off), wdims, wstrides,
-                wbox, westr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                wbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return TMAN_ERR_CUDA;
     }
-    // the output as 32 x 32 tiles in the 64-byte swizzle (the pair kernel's epilogue stores)
+    // the output as 32 x 32 tiles in the 64-byte swizzle (the epilogue's stores)
     CUtensorMap tmap_y;
     {
         const cuuint64_t ydims[2] = {(cuuint64_t)N, (cuuint64_t)M};
@@ -1064,9 +960,23 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
                 CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return TMAN_ERR_CUDA;
     }
-    if (bits == 2) return launch_bits<2>(tmap, tmap_w, tmap_y, p, mh, s);
-    if (bits == 3) return launch_bits<3>(tmap, tmap_w, tmap_y, p, mh, s);
-    return launch_bits<4>(tmap, tmap_w, tmap_y, p, mh, s);
+
+    uint8_t *w8 = static_cast<uint8_t *>(ws);
+    GemmParams p;
+    p.packed = pk;
+    p.planes = reinterpret_cast<const uint32_t *>(pk + L.planes_off);
+    p.scales = reinterpret_cast<const __half *>(pk + L.scales_off);
+    p.zeros = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
+    p.status = reinterpret_cast<uint32_t *>(w8);
+    p.flags = reinterpret_cast<uint32_t *>(w8 + kGemmFlagsOff);
+    p.partial = reinterpret_cast<float *>(w8 + kGemmPartialOff);
+    p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
+    p.tiles_m = (M + (pair ? 2 : 1) * rows_cta - 1) / ((pair ? 2 : 1) * rows_cta);
+    p.tiles_n = 0;             // set when the work is cut
+    p.whole_tiles = 1;
+    if (bits == 2) return launch_bits<2>(tmap_x, tmap_w, tmap_y, p, sms, s);
+    if (bits == 3) return launch_bits<3>(tmap_x, tmap_w, tmap_y, p, sms, s);
+    return launch_bits<4>(tmap_x, tmap_w, tmap_y, p, sms, s);
 }
 
 }  // namespace tman
