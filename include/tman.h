@@ -127,7 +127,14 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed /*host*/, c
 /* Prefill (paper Sec. 4.1 two-level LUT dequantization, Fig. 7; Sec. 4.2 three-stage pipeline,
  * Fig. 9): packed tiles are staged in shared memory, rebuilt into fp16 tiles through the
  * repack step and the per-(block, column) conversion table, and multiplied on the tensor
- * cores with fp32 accumulation.  M >= 1. */
+ * cores with fp32 accumulation.  M >= 1.
+ *   - The output is cut into tiles dealt to the SMs; when the tiles do not go round evenly the
+ *     k-range of the last ones is divided among the SMs and summed, in a fixed order, through
+ *     fp32 partial tiles in the workspace (tens of MB: ask tman_workspace_bytes(1, ...)).  The
+ *     result does not depend on timing: the same call gives the same bits.
+ *   - All CTAs of the call must be able to run at the same time (at most one per SM is
+ *     launched); if another kernel holds SMs for longer than a second while this one runs,
+ *     the call gives up with TMAN_ERR_TIMEOUT in the status word instead of waiting on. */
 tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream);
