@@ -54,8 +54,9 @@ template <int MH, bool PAIR> struct Cfg {
     static constexpr int TMEM_COLS = MH * BN;                         // one fp32 accumulator of BN columns per row block
     static constexpr int smem_bytes(int bits)
     {
-        // stages (multiples of 1 KB, so the staging tiles stay 1 KB aligned), staging, barriers, slack to align
-        return NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + bits * P_PLANE_BYTES) + NUM_EPI_WARPS * OUT_TILE_BYTES + 512 + 1024;
+        // stages (multiples of 1 KB, so the staging tiles stay 1 KB aligned), staging, barriers.  The kernel
+        // has no static shared memory, so the dynamic part starts 1 KB aligned (checked in the kernel).
+        return NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES + bits * P_PLANE_BYTES) + NUM_EPI_WARPS * OUT_TILE_BYTES + 512;
     }
 };
 
@@ -383,20 +384,19 @@ struct Span {
     long long full, Ur;        // tiles dealt whole; units of the remaining tiles
     long long next_whole;      // next whole tile of this worker
     int nu, W, w;
-    int npieces, piece;        // pieces of this worker's span, in walk order, and the next one
-    Segment pieces[3];
-    int first_late;            // pieces[first_late..] come after the whole tiles
+    Segment early, late;       // the piece this worker only contributes; the piece of the tile it finishes
+    bool has_early, has_late;
     __device__ Span(const GemmParams &p, int worker, int nworkers)
-        : nu(p.K / (2 * BK)), W(nworkers), w(worker), npieces(0), piece(0), first_late(0)
+        : nu(p.K / (2 * BK)), W(nworkers), w(worker), has_early(false), has_late(false)
     {
         const long long T = (long long)p.tiles_m * p.tiles_n;
         full = p.whole_tiles ? T : (T / nworkers) * nworkers;
         Ur = (T - full) * nu;
         next_whole = worker;
         long long lo = Ur * worker / nworkers, hi = Ur * (worker + 1) / nworkers;
-        Segment early[3], late[3];
-        int ne = 0, nl = 0;
-        while (hi > lo && ne + nl < 3) {               // from the last tile of the span to the first
+        // the span is at most one tile long: at most one piece that ends inside its tile (the last
+        // one) and one that reaches its tile's end
+        for (int i = 0; i < 2 && hi > lo; ++i) {       // from the last tile of the span to the first
             const long long tile = (hi - 1) / nu, t0 = tile * nu;
             const long long k0 = (lo > t0) ? lo - t0 : 0, k1 = hi - t0;
             Segment s;
@@ -405,17 +405,14 @@ struct Span {
             s.kb1 = 2 * (int)k1;
             s.whole = (k0 == 0 && k1 == nu);
             s.finishes = (k1 == nu);
-            if (s.finishes) late[nl++] = s;
-            else early[ne++] = s;
+            if (s.finishes) { late = s; has_late = true; }
+            else { early = s; has_early = true; }
             hi = t0 + k0;
         }
-        for (int i = 0; i < ne; ++i) pieces[npieces++] = early[i];
-        first_late = npieces;
-        for (int i = 0; i < nl; ++i) pieces[npieces++] = late[i];   // the tile this worker sums comes last
     }
     __device__ bool next(Segment &s)
     {
-        if (piece < first_late) { s = pieces[piece++]; return true; }
+        if (has_early) { s = early; has_early = false; return true; }
         if (next_whole < full) {
             s.tile = (int)next_whole;
             s.kb0 = 0;
@@ -424,7 +421,7 @@ struct Span {
             next_whole += W;
             return true;
         }
-        if (piece < npieces) { s = pieces[piece++]; return true; }
+        if (has_late) { s = late; has_late = false; return true; }
         return false;
     }
     // the worker that owns unit u of tile `tile` (one of the remaining tiles)
@@ -445,13 +442,16 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     constexpr int P_PLANE_BYTES = C::P_PLANE_BYTES, P_STAGE_BYTES = BITS * P_PLANE_BYTES, TMEM_COLS = C::TMEM_COLS;
     constexpr int ROWS_CTA = BM * MH;                  // token rows of a tile held by one CTA
     constexpr int NGROUP = PAIR ? 2 : 1;               // dequantization warp groups that take turns
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // in a pair, CTA 0 issues the MMAs and owns the shared barriers
     if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {   // same answer in every CTA
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
         return;
     }
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    if ((smem_u32(smem) & 1023u) != 0u) {              // the swizzled tiles need 1 KB alignment (same in every CTA)
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_CUDA);
+        return;
+    }
     uint8_t *a_tiles = smem;
     uint8_t *b_tiles = smem + NSTAGE * A_STAGE_BYTES;
     uint8_t *p_tiles = smem + NSTAGE * (A_STAGE_BYTES + B_STAGE_BYTES);
