@@ -358,9 +358,12 @@ def run_ours(args):
         print(json.dumps(line))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture exists)
-TRAFFIC_BYTES_PER_LAUNCH = None   # set from the ncu capture below
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
+# profiles/.  mpGEMV: one gate/up-sized launch moved 17.04 MB for 16.78 MB of algorithmic bytes
+# (+1.55 %); traffic grows with the bytes streamed, so the step's mean launch (25.17 MB) is scaled
+# by the same ratio.  mpGEMM: the M=1024, K=4096, N=14336 launch (the larger config-4 shape).
+TRAFFIC_BYTES_PER_LAUNCH = 25171968.0 * (17.04 / 16.78)
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 41.6e6
 
 
 def bench_gemm(torch, B, H, synth, peaks):
@@ -397,7 +400,7 @@ def bench_gemm(torch, B, H, synth, peaks):
     out["value"] = tf
     out["frac_of_nominal_fp16"] = tf / NOMINAL_FP16_TFLOPS
     out["roofline"] = {"bound": "tensor", "kernel": "mpgemm_kernel<4,2,true> (4-bit, CTA pairs, two row blocks per CTA)", "achieved": tf, "peak": peaks["tf_burst"],
-                       "unit": "TFLOP/s", "frac": tf / peaks["tf_burst"], "traffic": None,
+                       "unit": "TFLOP/s", "frac": tf / peaks["tf_burst"], "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
                        "peak_source": f"of {peaks['src']} (bf16 burst; fp16 has the same nominal rate)"}
     return out
 
