@@ -176,6 +176,13 @@ tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int g
  * device routine the decode kernel builds its tables from (paper Sec. 2.2). */
 tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_stream_t stream);
 
+/* How tman_mpgemm would cut a call's work on the current device (host-side decision, nothing is
+ * launched; no counterpart in the paper).  out6 (host) receives: 1 if pairs of CTAs work on a tile
+ * else 0; 128-token row blocks per CTA; row tiles; column tiles; 1 if every tile is dealt whole,
+ * 0 if the last tiles' k-range is divided among the workers and summed through the workspace;
+ * workers (CTAs or pairs) launched.  Tests use it to know that a shape takes the split path. */
+tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out6 /*host*/);
+
 #ifdef __cplusplus
 }
 #endif

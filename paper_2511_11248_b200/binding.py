@@ -22,7 +22,7 @@ OP_GEMV, OP_GEMM, OP_AUX = 0, 1, 2
 EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
-    "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_mpgemv_static", "tman_mpgemv_grouped",
+    "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
 ]
 
 _lib = None
@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
         L.tman_mpgemv_grouped.argtypes = [i, C.POINTER(vp), C.POINTER(sz), vp, C.POINTER(vp), i, i, C.POINTER(i), i, i, vp, sz, vp]
         L.tman_debug_indices.argtypes = [vp, i, i, i, i, vp, vp, sz, vp]
         L.tman_debug_luts.argtypes = [vp, i, i, vp, vp]
+        L.tman_debug_gemm_plan.argtypes = [i, i, i, i, i, C.POINTER(C.c_int)]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -161,6 +162,12 @@ def tman_debug_indices(packed, K, N, bits, group, idx, workspace, stream=None) -
     _check(lib().tman_debug_indices(_ptr(packed), K, N, bits, group, _ptr(idx), _ptr(workspace),
                                     workspace.numel() * workspace.element_size(), _stream(stream)),
            "tman_debug_indices")
+
+
+def tman_debug_gemm_plan(M, K, N, bits, group) -> dict:
+    out = (C.c_int * 6)()
+    _check(lib().tman_debug_gemm_plan(M, K, N, bits, group, out), "tman_debug_gemm_plan")
+    return dict(zip(("pair", "row_blocks", "tiles_m", "tiles_n", "whole_tiles", "workers"), list(out)))
 
 
 def tman_debug_luts(x, M, K, lut, stream=None) -> None:

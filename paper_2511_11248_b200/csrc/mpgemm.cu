@@ -441,7 +441,6 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     constexpr int NCTA = C::NCTA, NSTAGE = C::NSTAGE, A_STAGE_BYTES = C::A_STAGE_BYTES, B_STAGE_BYTES = C::B_STAGE_BYTES;
     constexpr int P_PLANE_BYTES = C::P_PLANE_BYTES, P_STAGE_BYTES = BITS * P_PLANE_BYTES, TMEM_COLS = C::TMEM_COLS;
     constexpr int ROWS_CTA = BM * MH;                  // token rows of a tile held by one CTA
-    constexpr int NGROUP = PAIR ? 2 : 1;               // dequantization warp groups that take turns
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // in a pair, CTA 0 issues the MMAs and owns the shared barriers
     if (!header_matches(p.packed, p.K, p.N, p.bits, p.group)) {   // same answer in every CTA
@@ -574,25 +573,27 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // ---- stage 2: two-level lookup dequantization of this CTA's channels ----------------------
         // A warp owns 16 channels and both plane words of a k-block: lane = (strip of the warp, word,
         // column of the strip).  With this split the 32 lanes read 32 different banks of the staged
-        // plane words and write eight different 16-byte bank groups per quarter-warp.  A CTA of a pair
-        // has 128 channels: the two halves of its sixteen warps take turns, two k-blocks each.
+        // plane words and write eight different 16-byte bank groups per quarter-warp.  When a CTA has at
+        // most 128 channels of a tile (always in a pair), eight warps cover them: the two halves of the
+        // sixteen warps then take turns, two k-blocks each.
         const int wd16 = warp - 2;
-        const int wd = wd16 % (NUM_DEQ_WARPS / NGROUP), grp = wd16 / (NUM_DEQ_WARPS / NGROUP);
         const int sl = lane >> 3, v = (lane >> 2) & 1, c = lane & 3;
         const int nblk = p.K / p.group;
         const int gshift = (p.group == 32) ? 5 : (p.group == 64) ? 6 : 7;
         auto block_of = [&](int kb) { return ((2 * kb + v) * 32) >> gshift; };
-        const int n_local = wd * 16 + sl * 4 + c;
-        const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
-        const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
-        const uint32_t xr = (uint32_t)(n_local & 7);
-        const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
-        // k-blocks this warp works on, by pipeline position (segments start at even k-blocks)
-        auto mine = [&](uint32_t it) { return NGROUP == 1 || (int)((it >> 1) & 1u) == grp; };
 
         uint32_t it = 0;
         while (ok && span.next(sg)) {
             const int chans = tile_bn(sg.tile) / NCTA;
+            const int ngroup = (PAIR || chans <= BN / 2) ? 2 : 1;
+            const int wd = wd16 % (NUM_DEQ_WARPS / ngroup), grp = wd16 / (NUM_DEQ_WARPS / ngroup);
+            const int n_local = wd * 16 + sl * 4 + c;
+            const uint32_t p_off = (uint32_t)(wd * 4 + sl) * 32u + (uint32_t)v * 16u + (uint32_t)c * 4u;
+            const uint32_t row_off = (uint32_t)(n_local >> 3) * 1024u + (uint32_t)(n_local & 7) * 128u;
+            const uint32_t xr = (uint32_t)(n_local & 7);
+            const uint32_t p_base = smem_u32(p_tiles) + p_off, b_base = smem_u32(b_tiles) + row_off;
+            // k-blocks this warp works on, by pipeline position (segments start at even k-blocks)
+            auto mine = [&](uint32_t i) { return ngroup == 1 || (int)((i >> 1) & 1u) == grp; };
             const int n = tile_col0(sg.tile) + (int)rank * chans + n_local;
             const bool valid = n_local < chans && n < p.N;   // channels past the tile are not used by the MMA
             const int nb = n >> 2;
@@ -622,7 +623,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         T.build(sv_next, zz_next);
                     }
                     // scale and zero-point of the block after this one are fetched one k-block ahead
-                    const int kn = (NGROUP == 1 || !(kb & 1)) ? kb + 1 : kb + 3;
+                    const int kn = (ngroup == 1 || !(kb & 1)) ? kb + 1 : kb + 3;
                     const int Bn = block_of(kn);
                     if (kn < sg.kb1 && Bn != cur_B && Bn != next_B) {
                         next_B = Bn;
@@ -830,55 +831,72 @@ EncodeTiledFn encode_fn()
 inline int gemm_mh(int M) { return M > 2 * BM ? 2 : 1; }
 inline bool gemm_pair(int M) { return M > BM; }
 
+// How a call's work is cut (host).  One worker per SM (pair of SMs), fewer when there is less work
+// than that.  The channels are cut into column tiles of almost equal width (multiples of 32, at
+// most 256) and the tiles dealt whole; the number of column tiles is the one with the least
+// estimated time for the longest worker: rounds of tiles x k-blocks x time of a k-block, which for
+// a pair hardly falls below 192 channels (the MMA's activation operand bounds it) and for a single
+// CTA is a latency chain plus the dequantization's share, in proportion to the width (measured
+// figures, microseconds: pair 0.74 / 0.76 / 0.87 at 128 / 192 / 256 channels, single CTA 0.51 / 0.59 /
+// 0.77 / 1.11 at 32 / 64 / 128 / 256).  The
+// alternative: the widest tiles, whole as far as they go round and the rest in equal spans, whose
+// split tiles cost their workers a partial tile written to and read back from the workspace (an SM
+// writes about 50 GB/s; the more pieces per tile, the more to read back).
+struct GemmPlan { int pair, mh, tiles_m, tiles_n, whole_tiles, workers; };
+
+GemmPlan plan_gemm(int M, int K, int N, int sms)
+{
+    GemmPlan g;
+    g.pair = gemm_pair(M) ? 1 : 0;
+    g.mh = gemm_mh(M);
+    const int ncta = g.pair ? 2 : 1, rows = ncta * BM * g.mh;
+    g.tiles_m = (M + rows - 1) / rows;
+    const long long nu = K / (2 * BK);
+    long long workers = (sms < kMaxGemmCtas ? sms : kMaxGemmCtas) / ncta;
+    if (workers < 1) workers = 1;
+    const int n32 = (N + 31) / 32, tn_min = (n32 + BN / 32 - 1) / (BN / 32);
+    const bool pair = g.pair != 0;
+    auto kb_us = [pair](int width) {
+        const double w = (double)width;
+        if (pair) return w <= 192 ? 0.70 + 0.0003 * w : 0.7576 + 0.00175 * (w - 192);
+        return 0.42 + 0.0027 * w;
+    };
+    double best = 1e300;
+    g.whole_tiles = 1;
+    g.tiles_n = tn_min;
+    for (int tn = tn_min; tn <= n32 && tn <= 8 * tn_min; ++tn) {
+        const long long rounds = ((long long)g.tiles_m * tn + workers - 1) / workers;
+        const int wmax = 32 * ((n32 + tn - 1) / tn);
+        const double cost = (double)rounds * (2.0 * nu * kb_us(wmax) + 3.0);
+        if (cost <= best + 1e-9) { best = cost; g.tiles_n = tn; }     // ties: more, narrower tiles
+    }
+    {
+        const long long t = (long long)g.tiles_m * tn_min, rest = t % workers;
+        const double cost = (double)(t / workers) * (2.0 * nu * kb_us(BN) + 3.0) +
+                            (double)((rest * nu + workers - 1) / workers) * 2.0 * kb_us(BN) +
+                            (rest ? (pair ? 24.0 : 16.0) + 3.0 * (double)workers / (double)rest : 0.0);
+        if (rest != 0 && cost < best) {
+            g.whole_tiles = 0;
+            g.tiles_n = tn_min;
+        }
+    }
+    const long long tiles = (long long)g.tiles_m * g.tiles_n;
+    if (tiles < workers) {                             // fewer tiles than workers: as many workers as units at most
+        const long long units = g.whole_tiles ? tiles : tiles * nu;
+        if (workers > units) workers = units;
+    }
+    g.workers = (int)workers;
+    return g;
+}
+
 template <int BITS, int MH, bool PAIR>
 tman_status launch_cfg(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const GemmParams &p,
-                       int sms, cudaStream_t s)
+                       int workers, cudaStream_t s)
 {
     using C = Cfg<MH, PAIR>;
     auto kern = mpgemm_kernel<BITS, MH, PAIR>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes(BITS)) != cudaSuccess)
         return TMAN_ERR_CUDA;
-    // One worker per SM (pair of SMs), fewer when there is less work than that.  The channels are cut
-    // into column tiles of almost equal width (multiples of 32, at most 256) and the tiles dealt whole;
-    // the number of column tiles is the one with the least estimated time for the longest worker:
-    // rounds of tiles x k-blocks x time of a k-block, which for a pair hardly falls below 192 channels
-    // (the MMA's activation operand bounds it) and for a single CTA is the dequantization's, in
-    // proportion to the width (measured figures, microseconds).  The alternative: the widest tiles,
-    // whole as far as they go round and the rest in equal spans, whose split tiles cost their workers a
-    // partial tile written to and read back from the workspace (an SM writes about 50 GB/s).
-    const long long nu = p.K / (2 * BK);
-    long long workers = (sms < kMaxGemmCtas ? sms : kMaxGemmCtas) / C::NCTA;
-    if (workers < 1) return TMAN_ERR_CUDA;
-    GemmParams q = p;
-    const int n32 = (p.N + 31) / 32, tn_min = (n32 + BN / 32 - 1) / (BN / 32);
-    auto kb_us = [](int width) {
-        const double w = (double)width;
-        return PAIR ? (0.0034 * w > 0.74 ? 0.0034 * w : 0.74) : (1.1 * w / 256 > 0.3 ? 1.1 * w / 256 : 0.3);
-    };
-    double best = 1e300;
-    q.whole_tiles = 1;
-    q.tiles_n = tn_min;
-    for (int tn = tn_min; tn <= n32 && tn <= 8 * tn_min; ++tn) {
-        const long long rounds = ((long long)p.tiles_m * tn + workers - 1) / workers;
-        const int wmax = 32 * ((n32 + tn - 1) / tn);
-        const double cost = (double)rounds * (2.0 * nu * kb_us(wmax) + 3.0);
-        if (cost < best - 1e-9) { best = cost; q.tiles_n = tn; }
-    }
-    {
-        const long long t = (long long)p.tiles_m * tn_min, rest = t % workers;
-        const double cost = (double)(t / workers) * (2.0 * nu * kb_us(BN) + 3.0) +
-                            (double)((rest * nu + workers - 1) / workers) * 2.0 * kb_us(BN) +
-                            (rest ? (PAIR ? 24.0 : 16.0) + 3.0 * (double)workers / (double)rest : 0.0);   // more pieces per tile: more to read back
-        if (rest != 0 && cost < best) {
-            q.whole_tiles = 0;
-            q.tiles_n = tn_min;
-        }
-    }
-    const long long tiles = (long long)q.tiles_m * q.tiles_n;
-    if (tiles < workers) {                             // fewer tiles than workers: as many workers as units at most
-        const long long units = q.whole_tiles ? tiles : tiles * nu;
-        if (workers > units) workers = units;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(workers * C::NCTA));
     cfg.blockDim = dim3(GEMM_THREADS);
@@ -891,20 +909,29 @@ tman_status launch_cfg(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, con
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, q) != cudaSuccess) return TMAN_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, p) != cudaSuccess) return TMAN_ERR_CUDA;
     return TMAN_OK;
 }
 
 template <int BITS>
 tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const GemmParams &p,
-                        int sms, cudaStream_t s)
+                        const GemmPlan &g, cudaStream_t s)
 {
-    if (!gemm_pair(p.M)) return launch_cfg<BITS, 1, false>(tmap_x, tmap_w, tmap_y, p, sms, s);
-    if (gemm_mh(p.M) == 1) return launch_cfg<BITS, 1, true>(tmap_x, tmap_w, tmap_y, p, sms, s);
-    return launch_cfg<BITS, 2, true>(tmap_x, tmap_w, tmap_y, p, sms, s);
+    if (!g.pair) return launch_cfg<BITS, 1, false>(tmap_x, tmap_w, tmap_y, p, g.workers, s);
+    if (g.mh == 1) return launch_cfg<BITS, 1, true>(tmap_x, tmap_w, tmap_y, p, g.workers, s);
+    return launch_cfg<BITS, 2, true>(tmap_x, tmap_w, tmap_y, p, g.workers, s);
 }
 
 }  // namespace
+
+tman_status mpgemm_plan(int M, int K, int N, int *out6)
+{
+    const int sms = sm_count();
+    if (sms <= 0) return TMAN_ERR_CUDA;
+    const GemmPlan g = plan_gemm(M, K, N, sms);
+    out6[0] = g.pair; out6[1] = g.mh; out6[2] = g.tiles_m; out6[3] = g.tiles_n; out6[4] = g.whole_tiles; out6[5] = g.workers;
+    return TMAN_OK;
+}
 
 size_t mpgemm_workspace_bytes(int M, int, int)
 {
@@ -919,9 +946,9 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     if (!enc) return TMAN_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
-    const int mh = gemm_mh(M);
-    const bool pair = gemm_pair(M);
-    const int rows_cta = BM * mh, bn_cta = pair ? BN / 2 : BN;
+    const GemmPlan g = plan_gemm(M, K, N, sms);
+    const bool pair = g.pair != 0;
+    const int rows_cta = BM * g.mh, bn_cta = pair ? BN / 2 : BN;
     const cuuint32_t estr[3] = {1, 1, 1};
 
     // activations: boxes of one k-block x a CTA's token rows, 128-byte swizzle
@@ -971,12 +998,12 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.flags = reinterpret_cast<uint32_t *>(w8 + kGemmFlagsOff);
     p.partial = reinterpret_cast<float *>(w8 + kGemmPartialOff);
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
-    p.tiles_m = (M + (pair ? 2 : 1) * rows_cta - 1) / ((pair ? 2 : 1) * rows_cta);
-    p.tiles_n = 0;             // set when the work is cut
-    p.whole_tiles = 1;
-    if (bits == 2) return launch_bits<2>(tmap_x, tmap_w, tmap_y, p, sms, s);
-    if (bits == 3) return launch_bits<3>(tmap_x, tmap_w, tmap_y, p, sms, s);
-    return launch_bits<4>(tmap_x, tmap_w, tmap_y, p, sms, s);
+    p.tiles_m = g.tiles_m;
+    p.tiles_n = g.tiles_n;
+    p.whole_tiles = g.whole_tiles;
+    if (bits == 2) return launch_bits<2>(tmap_x, tmap_w, tmap_y, p, g, s);
+    if (bits == 3) return launch_bits<3>(tmap_x, tmap_w, tmap_y, p, g, s);
+    return launch_bits<4>(tmap_x, tmap_w, tmap_y, p, g, s);
 }
 
 }  // namespace tman

@@ -64,6 +64,31 @@ def test_pair_kernel_cases(M, K, N, bits, G):
     check_full(synth.small_case(M, K, N, bits, G, seed=M + K + N + bits, outliers=(bits == 4)))
 
 
+# Long K and few tiles: the last tiles' k-blocks are divided among the workers and summed through
+# the workspace (many pieces per tile).  Pairs of CTAs with two and one row block, a single CTA,
+# ragged M and N, every bit width; compared element by element.
+SPLIT = [(300, 8192, 1024, 4, 128), (520, 8192, 1288, 2, 64), (200, 16384, 520, 3, 128), (100, 24576, 2560, 3, 128)]
+
+
+@pytest.mark.parametrize("M,K,N,bits,G", SPLIT)
+def test_split_tile_cases(M, K, N, bits, G):
+    plan = B.tman_debug_gemm_plan(M, K, N, bits, G)
+    assert plan["whole_tiles"] == 0, plan          # the shape must take the path this test is about
+    c = synth.small_case(M, K, N, bits, G, seed=M + K + N + bits)
+    check_full(c)
+    # the same call again on the same workspace: flags and partial tiles were left ready
+    dev = H.device_case(c)
+    packed = H.pack_case(c, dev)
+    ws = H.alloc_workspace(B.OP_GEMM, c.M, c.K, c.N, c.bits, c.group)
+    ys = []
+    for _ in range(3):
+        y = torch.full((c.M, c.N), float("nan"), dtype=torch.float16, device="cuda")
+        B.tman_mpgemm(packed, dev["x"], y, c.M, c.K, c.N, c.bits, c.group, ws)
+        ys.append(y)
+    assert B.tman_read_status(ws) == 0
+    assert torch.equal(ys[0], ys[1]) and torch.equal(ys[1], ys[2])   # fixed summation order: same bits
+
+
 def test_integer_case_is_exact():
     rng = np.random.default_rng(5)
     c = synth.small_case(130, 512, 136, 3, 64, seed=31)
