@@ -77,7 +77,8 @@ struct GemmParams {
     float          *partial;
     int M, K, N, bits, group;
     int tiles_m, tiles_n;
-    int whole_tiles;           // spans are whole tiles (no tile is split)
+    int span_tiles;            // the last span_tiles tiles are dealt as equal spans of k-blocks (0: every tile whole)
+    int col_fastest;           // tile number = row tile * tiles_n + column tile (else column tile * tiles_m + row tile)
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -369,34 +370,32 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
 }
 
 // ---- split of the work ----------------------------------------------------------------------
-// T tiles (row tile fastest), W workers.  The first floor(T / W) * W tiles are dealt whole, round-robin.
-// The k-blocks of the remaining tiles (fewer than W), laid end to end in units of two k-blocks (a
-// 128-wide quantization block is never cut), are dealt in equal contiguous spans, so every worker is
-// busy to the end whatever the shape.  A span is shorter than a tile: it is a piece of one tile or the
-// end of one and the start of the next.  A tile cut into several pieces ("split tile") is summed by
-// the worker that owns its last unit: the others, which all have lower numbers, write their fp32
-// accumulators to the workspace and raise a flag.  A worker's walk: first the piece that it only
-// contributes (so that it is ready long before it is needed), then its whole tiles, last the piece
-// of the tile that it finishes.  (whole_tiles: all T tiles are dealt whole.)
+// T tiles (row tile fastest), W workers.  The first `whole` tiles (a multiple of W) are dealt whole,
+// round-robin.  The k-blocks of the remaining tiles (fewer than 2 W), laid end to end in units of two
+// k-blocks (a 128-wide quantization block is never cut), are dealt in equal contiguous spans, so
+// every worker is busy to the end whatever the shape.  A span is shorter than two tiles: at most
+// the end of one tile, one whole tile and the start of the next.  A tile cut into several pieces
+// ("split tile") is summed by the worker that owns its last unit: the others, which all have lower
+// numbers, write their fp32 accumulators to the workspace and raise a flag.  A worker's walk: first
+// the piece that it only contributes (so that it is ready long before it is needed), then its whole
+// tiles, last the piece of the tile that it finishes.
 struct Segment { int tile, kb0, kb1; bool whole, finishes; };
 
 struct Span {
-    long long full, Ur;        // tiles dealt whole; units of the remaining tiles
-    long long next_whole;      // next whole tile of this worker
+    long long full, Ur;        // tiles dealt whole round-robin; units of the remaining tiles
+    long long next_whole;      // next round-robin tile of this worker
     int nu, W, w;
-    Segment early, late;       // the piece this worker only contributes; the piece of the tile it finishes
-    bool has_early, has_late;
+    Segment early, mid, late;  // the piece this worker only contributes; a whole tile of its span; the piece it finishes
+    bool has_early, has_mid, has_late;
     __device__ Span(const GemmParams &p, int worker, int nworkers)
-        : nu(p.K / (2 * BK)), W(nworkers), w(worker), has_early(false), has_late(false)
+        : nu(p.K / (2 * BK)), W(nworkers), w(worker), has_early(false), has_mid(false), has_late(false)
     {
         const long long T = (long long)p.tiles_m * p.tiles_n;
-        full = p.whole_tiles ? T : (T / nworkers) * nworkers;
-        Ur = (T - full) * nu;
+        full = T - p.span_tiles;
+        Ur = (long long)p.span_tiles * nu;
         next_whole = worker;
         long long lo = Ur * worker / nworkers, hi = Ur * (worker + 1) / nworkers;
-        // the span is at most one tile long: at most one piece that ends inside its tile (the last
-        // one) and one that reaches its tile's end
-        for (int i = 0; i < 2 && hi > lo; ++i) {       // from the last tile of the span to the first
+        for (int i = 0; i < 3 && hi > lo; ++i) {       // from the last tile of the span to the first
             const long long tile = (hi - 1) / nu, t0 = tile * nu;
             const long long k0 = (lo > t0) ? lo - t0 : 0, k1 = hi - t0;
             Segment s;
@@ -405,7 +404,8 @@ struct Span {
             s.kb1 = 2 * (int)k1;
             s.whole = (k0 == 0 && k1 == nu);
             s.finishes = (k1 == nu);
-            if (s.finishes) { late = s; has_late = true; }
+            if (s.whole) { mid = s; has_mid = true; }
+            else if (s.finishes) { late = s; has_late = true; }
             else { early = s; has_early = true; }
             hi = t0 + k0;
         }
@@ -421,6 +421,7 @@ struct Span {
             next_whole += W;
             return true;
         }
+        if (has_mid) { s = mid; has_mid = false; return true; }
         if (has_late) { s = late; has_late = false; return true; }
         return false;
     }
@@ -504,12 +505,16 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     Segment sg;
     // a tile's place in the output, the channels this CTA dequantizes (a pair halves the tile's channels;
     // the last tile of a row may be narrower: a multiple of 32 channels that reaches N)
-    auto tile_rows = [&](int tile) { return (tile % p.tiles_m) * (NCTA * ROWS_CTA) + (int)rank * ROWS_CTA; };
+    // Tiles with consecutive numbers run at the same time; the host numbers them so that a round of
+    // tiles touches the fewest bytes (row tiles of activations, column tiles of packed weights).
+    auto tile_tm = [&](int tile) { return p.col_fastest ? tile / p.tiles_n : tile % p.tiles_m; };
+    auto tile_ct = [&](int tile) { return p.col_fastest ? tile % p.tiles_n : tile / p.tiles_m; };
+    auto tile_rows = [&](int tile) { return tile_tm(tile) * (NCTA * ROWS_CTA) + (int)rank * ROWS_CTA; };
     // (the N/32 column units are cut into tiles_n column tiles of almost equal width, at most BN)
     const int n32 = (p.N + 31) / 32;
     auto tile_unit0 = [&](int ct) { return (int)(((long long)n32 * ct) / p.tiles_n); };
-    auto tile_col0 = [&](int tile) { return 32 * tile_unit0(tile / p.tiles_m); };
-    auto tile_bn = [&](int tile) { const int ct = tile / p.tiles_m; return 32 * (tile_unit0(ct + 1) - tile_unit0(ct)); };
+    auto tile_col0 = [&](int tile) { return 32 * tile_unit0(tile_ct(tile)); };
+    auto tile_bn = [&](int tile) { const int ct = tile_ct(tile); return 32 * (tile_unit0(ct + 1) - tile_unit0(ct)); };
     const uint32_t full_lead = PAIR ? mapa_u32(full0, 0) : full0, acce_lead = PAIR ? mapa_u32(acce, 0) : acce;
     auto arrive_lead = [&](uint32_t bar) {
         if constexpr (PAIR) mbar_arrive_cluster(bar);
@@ -842,9 +847,9 @@ inline bool gemm_pair(int M) { return M > BM; }
 // alternative: the widest tiles, whole as far as they go round and the rest in equal spans, whose
 // split tiles cost their workers a partial tile written to and read back from the workspace (an SM
 // writes about 50 GB/s; the more pieces per tile, the more to read back).
-struct GemmPlan { int pair, mh, tiles_m, tiles_n, whole_tiles, workers; };
+struct GemmPlan { int pair, mh, tiles_m, tiles_n, span_tiles, workers, col_fastest; };
 
-GemmPlan plan_gemm(int M, int K, int N, int sms)
+GemmPlan plan_gemm(int M, int K, int N, int bits, int sms)
 {
     GemmPlan g;
     g.pair = gemm_pair(M) ? 1 : 0;
@@ -862,7 +867,7 @@ GemmPlan plan_gemm(int M, int K, int N, int sms)
         return 0.42 + 0.0027 * w;
     };
     double best = 1e300;
-    g.whole_tiles = 1;
+    g.span_tiles = 0;
     g.tiles_n = tn_min;
     for (int tn = tn_min; tn <= n32 && tn <= 8 * tn_min; ++tn) {
         const long long rounds = ((long long)g.tiles_m * tn + workers - 1) / workers;
@@ -871,21 +876,31 @@ GemmPlan plan_gemm(int M, int K, int N, int sms)
         if (cost <= best + 1e-9) { best = cost; g.tiles_n = tn; }     // ties: more, narrower tiles
     }
     {
+        // widest tiles; the remainder of the last round is cut into spans, together with one whole
+        // round when the remainder alone would be cut into many pieces per tile
         const long long t = (long long)g.tiles_m * tn_min, rest = t % workers;
-        const double cost = (double)(t / workers) * (2.0 * nu * kb_us(BN) + 3.0) +
-                            (double)((rest * nu + workers - 1) / workers) * 2.0 * kb_us(BN) +
-                            (rest ? (pair ? 24.0 : 16.0) + 3.0 * (double)workers / (double)rest : 0.0);
-        if (rest != 0 && cost < best) {
-            g.whole_tiles = 0;
+        const long long span = (rest != 0 && rest < workers / 2 && t > workers) ? rest + workers : rest;
+        const double cost = (double)((t - span) / workers) * (2.0 * nu * kb_us(BN) + 3.0) +
+                            (double)((span * nu + workers - 1) / workers) * 2.0 * kb_us(BN) +
+                            (span ? (pair ? 24.0 : 16.0) + 3.0 * (double)workers / (double)span : 0.0);
+        if (span != 0 && cost < best) {
+            g.span_tiles = (int)span;
             g.tiles_n = tn_min;
         }
     }
     const long long tiles = (long long)g.tiles_m * g.tiles_n;
     if (tiles < workers) {                             // fewer tiles than workers: as many workers as units at most
-        const long long units = g.whole_tiles ? tiles : tiles * nu;
+        const long long units = g.span_tiles ? tiles * nu : tiles;
         if (workers > units) workers = units;
     }
     g.workers = (int)workers;
+    // tile numbering: bytes a round of `workers` consecutive tiles touches, either way
+    {
+        const double a_tile = (double)rows * K * 2.0, b_tile = (double)N / g.tiles_n * K * bits / 8.0;
+        const long long rows_r = g.tiles_m < workers ? g.tiles_m : workers, cols_r = (workers + g.tiles_m - 1) / g.tiles_m;
+        const long long cols_c = g.tiles_n < workers ? g.tiles_n : workers, rows_c = (workers + g.tiles_n - 1) / g.tiles_n;
+        g.col_fastest = (rows_c * a_tile + cols_c * b_tile < rows_r * a_tile + cols_r * b_tile) ? 1 : 0;
+    }
     return g;
 }
 
@@ -928,8 +943,8 @@ tman_status mpgemm_plan(int M, int K, int N, int *out6)
 {
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
-    const GemmPlan g = plan_gemm(M, K, N, sms);
-    out6[0] = g.pair; out6[1] = g.mh; out6[2] = g.tiles_m; out6[3] = g.tiles_n; out6[4] = g.whole_tiles; out6[5] = g.workers;
+    const GemmPlan g = plan_gemm(M, K, N, 4, sms);
+    out6[0] = g.pair; out6[1] = g.mh; out6[2] = g.tiles_m; out6[3] = g.tiles_n; out6[4] = g.span_tiles ? 0 : 1; out6[5] = g.workers;
     return TMAN_OK;
 }
 
@@ -946,7 +961,7 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     if (!enc) return TMAN_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
-    const GemmPlan g = plan_gemm(M, K, N, sms);
+    const GemmPlan g = plan_gemm(M, K, N, bits, sms);
     const bool pair = g.pair != 0;
     const int rows_cta = BM * g.mh, bn_cta = pair ? BN / 2 : BN;
     const cuuint32_t estr[3] = {1, 1, 1};
@@ -1000,7 +1015,8 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
     p.tiles_m = g.tiles_m;
     p.tiles_n = g.tiles_n;
-    p.whole_tiles = g.whole_tiles;
+    p.span_tiles = g.span_tiles;
+    p.col_fastest = g.col_fastest;
     if (bits == 2) return launch_bits<2>(tmap_x, tmap_w, tmap_y, p, g, s);
     if (bits == 3) return launch_bits<3>(tmap_x, tmap_w, tmap_y, p, g, s);
     return launch_bits<4>(tmap_x, tmap_w, tmap_y, p, g, s);
