@@ -2,11 +2,13 @@
 // (paper Sec. 4.1 "Unified Layout through Fused LUT-based Dequantization", Fig. 7;
 //  Sec. 4.2 "Pipelining to Hide Dequantization Overhead", Fig. 9).
 //
-// The output is cut into tiles of 256 channels x 128*MH tokens (one CTA, at most 128 tokens) or
-// 256*MH tokens (a pair of CTAs on two SMs).  A tile's work is its K/64 k-blocks; the k-blocks of all
-// tiles, laid end to end, are dealt to the workers (CTAs or pairs, one per SM or SM pair) in equal
-// contiguous spans, so every SM is busy to the end whatever the shape.  A tile whose k-blocks fall
-// into several spans is summed through fp32 partial tiles in the workspace (see "split tiles").
+// The output is cut into tiles of up to 256 channels x 128*MH tokens (one CTA, at most 128 tokens) or
+// 256*MH tokens (a pair of CTAs on two SMs).  A tile's work is its K/64 k-blocks.  The host chooses
+// how many column tiles there are and deals the tiles to the workers (CTAs or pairs, at most one per
+// SM or SM pair), whole as far as they go round; where whole tiles would leave SMs idle, the
+// k-blocks of the last tiles are laid end to end and dealt in equal spans, and a tile whose
+// k-blocks fall into several spans is summed through fp32 partial tiles in the workspace (see
+// "split of the work").
 // Four kinds of agents run concurrently on a ring of shared-memory stages guarded by mbarriers (the
 // paper's DMA / vector-core / matrix-core stages):
 //   * warp 0, one lane : TMA loads of the fp16 activation tile (128-byte swizzle) and of the packed
