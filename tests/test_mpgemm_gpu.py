@@ -100,6 +100,31 @@ def test_integer_case_is_exact():
     assert np.array_equal(got, want.astype(np.float16).astype(np.float64))
 
 
+def test_pair_kernel_refuses_a_foreign_buffer_and_a_small_workspace():
+    """Enough tokens for CTA pairs: both CTAs of every cluster must leave cleanly on a header mismatch."""
+    M, K, N, bits, G = 600, 512, 1024, 4, 128
+    c = synth.small_case(M, K, N, bits, G, seed=77)
+    dev = H.device_case(c)
+    junk = torch.zeros(B.tman_packed_bytes(K, N, bits, G), dtype=torch.uint8, device="cuda")
+    ws = H.alloc_workspace(B.OP_GEMM, M, K, N, bits, G)
+    y = torch.full((M, N), 3.0, dtype=torch.float16, device="cuda")
+    B.tman_mpgemm(junk, dev["x"], y, M, K, N, bits, G, ws)
+    assert B.tman_read_status(ws) == 5          # TMAN_ERR_BAD_PACKED
+    assert bool((y == 3.0).all())
+    # the library is usable afterwards, on a freshly prepared workspace
+    B.tman_workspace_init(ws)
+    packed = H.pack_case(c, dev)
+    B.tman_mpgemm(packed, dev["x"], y, M, K, N, bits, G, ws)
+    assert B.tman_read_status(ws) == 0
+    ref = orc.mpgemm(c.x, c.codes, c.scales, c.zeros, c.group)
+    assert float(np.max(np.abs(H.to_f64(y) - ref)) / np.max(np.abs(ref))) <= TOL
+    # a workspace smaller than tman_workspace_bytes asks for is refused before any launch
+    small = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.TmanError) as e:
+        B.tman_mpgemm(packed, dev["x"], y, M, K, N, bits, G, small)
+    assert e.value.status == 4                  # TMAN_ERR_BUFFER_TOO_SMALL
+
+
 def test_gemm_and_gemv_read_the_same_packed_buffer():
     c = synth.small_case(4, 1024, 264, 4, 64, seed=32)
     dev = H.device_case(c)
