@@ -8,6 +8,8 @@ grouped call, o, gate and up in one grouped call, down), replayed from a CUDA gr
 weight sets larger than L2; reports weight-stream GB/s of the layer (sum of bytes / sum of time).
 Config 5: one call per shape, rotating packed copies larger than L2; reports TFLOP/s.
 Synthetic seeded inputs (value distributions of the parity tests); one JSON line per case.
+With --dense every case also times the same product with fp16 weights through torch.matmul (the
+library GEMM/GEMV: a yardstick for "what the low-bit weights buy or cost", not part of the path).
 """
 from __future__ import annotations
 
@@ -38,6 +40,47 @@ def event_us(fn, reps):
         torch.cuda.synchronize()
         ts.append(e0.elapsed_time(e1) * 1e3)
     return float(np.median(ts))
+
+
+def dense_layer_us(M, reps):
+    """The layer's seven products with fp16 weights (torch.matmul), rotating weight sets > L2."""
+    layer_bytes = sum(K * N * 2 for _, K, N in LLAMA3_8B_LAYER)
+    nsets = max(2, int(2.2 * L2_BYTES // layer_bytes) + 1)
+    sets = [[(torch.randn((M, K), dtype=torch.float16, device="cuda"),
+              torch.randn((K, N), dtype=torch.float16, device="cuda") * 0.02) for _, K, N in LLAMA3_8B_LAYER]
+            for _ in range(nsets)]
+
+    def layer(e):
+        for x, w in e:
+            torch.matmul(x, w)
+
+    for e in sets:
+        layer(e)
+    torch.cuda.synchronize()
+    nrep = 4 * nsets
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(nrep):
+            layer(sets[i % nsets])
+    g.replay()
+    torch.cuda.synchronize()
+    return event_us(g.replay, reps) / nrep
+
+
+def dense_case_us(M, K, N, reps):
+    x = torch.randn((M, K), dtype=torch.float16, device="cuda")
+    ncopy = max(2, int(2.2 * L2_BYTES // (K * N * 2)) + 1)
+    ws = [torch.randn((K, N), dtype=torch.float16, device="cuda") * 0.02 for _ in range(ncopy)]
+    y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    for w in ws[:2]:
+        torch.matmul(x, w, out=y)
+    torch.cuda.synchronize()
+
+    def run():
+        for w in ws:
+            torch.matmul(x, w, out=y)
+
+    return event_us(run, reps) / ncopy
 
 
 def decode_layer(bits, group, M, reps):
@@ -109,18 +152,33 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", type=int, choices=[3, 5], required=True)
     ap.add_argument("--reps", type=int, default=7)
+    ap.add_argument("--dense", action="store_true", help="also time the fp16-weight product (torch.matmul)")
     a = ap.parse_args()
     if a.config == 3:
+        dense = {M: dense_layer_us(M, a.reps) for M in (1, 2, 4, 8)} if a.dense else {}
+        torch.cuda.empty_cache()
         for bits in (2, 3, 4):
             for M in (1, 2, 4, 8):
-                print(json.dumps(decode_layer(bits, 128, M, a.reps)), flush=True)
+                r = decode_layer(bits, 128, M, a.reps)
+                if a.dense:
+                    r["dense_fp16_layer_us"] = round(dense[M], 2)
+                    r["speedup_vs_dense_fp16"] = round(dense[M] / r["layer_us"], 2)
+                print(json.dumps(r), flush=True)
                 torch.cuda.empty_cache()
     else:
+        dense = {}
         for bits in (2, 4):
             for group in (64, 128):
                 for M in (128, 512, 2048, 8192):
                     for _, K, N in synth.QWEN25_7B_PROJ:
-                        print(json.dumps(prefill_case(M, K, N, bits, group, a.reps)), flush=True)
+                        r = prefill_case(M, K, N, bits, group, a.reps)
+                        if a.dense:
+                            if (M, K, N) not in dense:
+                                dense[(M, K, N)] = dense_case_us(M, K, N, a.reps)
+                                torch.cuda.empty_cache()
+                            r["dense_fp16_us"] = round(dense[(M, K, N)], 1)
+                            r["time_vs_dense_fp16"] = round(r["us"] / dense[(M, K, N)], 2)
+                        print(json.dumps(r), flush=True)
                         torch.cuda.empty_cache()
 
 
