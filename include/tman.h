@@ -128,10 +128,11 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed /*host*/, c
  * Fig. 9): packed tiles are staged in shared memory, rebuilt into fp16 tiles through the
  * repack step and the per-(block, column) conversion table, and multiplied on the tensor
  * cores with fp32 accumulation.  M >= 1.
- *   - The output is cut into tiles dealt to the SMs; when the tiles do not go round evenly the
- *     k-range of the last ones is divided among the SMs and summed, in a fixed order, through
- *     fp32 partial tiles in the workspace (tens of MB: ask tman_workspace_bytes(1, ...)).  The
- *     result does not depend on timing: the same call gives the same bits.
+ *   - The output is cut into tiles dealt to the SMs; when the tiles do not go round evenly, or
+ *     are too few to fill the machine, the k-range of tiles is divided among the SMs and summed,
+ *     in a fixed order, through fp32 partial tiles in the workspace (tens of MB: ask
+ *     tman_workspace_bytes(1, ...)).  The result does not depend on timing: the same call gives
+ *     the same bits.
  *   - All CTAs of the call must be able to run at the same time (at most one per SM is
  *     launched); if another kernel holds SMs for longer than a second while this one runs,
  *     the call gives up with TMAN_ERR_TIMEOUT in the status word instead of waiting on. */
@@ -177,11 +178,12 @@ tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int g
 tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_stream_t stream);
 
 /* How tman_mpgemm would cut a call's work on the current device (host-side decision, nothing is
- * launched; no counterpart in the paper).  out6 (host) receives: 1 if pairs of CTAs work on a tile
- * else 0; 128-token row blocks per CTA; row tiles; column tiles; 1 if every tile is dealt whole,
- * 0 if the last tiles' k-range is divided among the workers and summed through the workspace;
- * workers (CTAs or pairs) launched.  Tests use it to know that a shape takes the split path. */
-tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out6 /*host*/);
+ * launched; no counterpart in the paper).  out8 (host) receives: 1 if pairs of CTAs work on a tile
+ * else 0; 128-token row blocks per CTA; row tiles; column tiles; 1 if every tile is dealt whole
+ * else 0; workers (CTAs or pairs) launched; number of last tiles whose k-blocks are dealt as equal
+ * spans (0: none); pieces every tile's k-blocks are split into (0: not split).  Tests use it to
+ * know which path a shape takes. */
+tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out8 /*host*/);
 
 #ifdef __cplusplus
 }

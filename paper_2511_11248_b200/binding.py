@@ -165,9 +165,9 @@ def tman_debug_indices(packed, K, N, bits, group, idx, workspace, stream=None) -
 
 
 def tman_debug_gemm_plan(M, K, N, bits, group) -> dict:
-    out = (C.c_int * 6)()
+    out = (C.c_int * 8)()
     _check(lib().tman_debug_gemm_plan(M, K, N, bits, group, out), "tman_debug_gemm_plan")
-    return dict(zip(("pair", "row_blocks", "tiles_m", "tiles_n", "whole_tiles", "workers"), list(out)))
+    return dict(zip(("pair", "row_blocks", "tiles_m", "tiles_n", "whole_tiles", "workers", "span_tiles", "pieces"), list(out)))
 
 
 def tman_debug_luts(x, M, K, lut, stream=None) -> None:

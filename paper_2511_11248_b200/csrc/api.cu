@@ -173,13 +173,13 @@ tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_st
     return launch_debug_luts(x_f16, M, K, lut, reinterpret_cast<cudaStream_t>(stream));
 }
 
-tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out6)
+tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out8)
 {
-    if (!out6) return TMAN_ERR_NULL;
+    if (!out8) return TMAN_ERR_NULL;
     tman_status st = check_format(K, N, bits, group);
     if (st != TMAN_OK) return st;
     if (M < 1) return TMAN_ERR_SHAPE;
-    return mpgemm_plan(M, K, N, out6);
+    return mpgemm_plan(M, K, N, out8);
 }
 
 }  // extern "C"

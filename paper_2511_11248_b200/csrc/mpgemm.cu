@@ -62,12 +62,15 @@ template <int MH, bool PAIR> struct Cfg {
     }
 };
 
-// Workspace: status word (kWsStatusBytes), one flag per epilogue warp of every CTA, then one fp32
-// partial tile per CTA (a worker writes at most one per launch).
+// Workspace: status word (kWsStatusBytes), one flag per epilogue warp of every CTA (spans), one flag
+// per (epilogue warp of a CTA, sending piece) (even split), then one fp32 partial tile per CTA (spans: a
+// worker writes at most one per launch; even split: the chunks the other pieces send to this CTA).
+constexpr int kMaxSplit = 8;                    // pieces of a tile in the even split
 constexpr size_t kGemmFlagsOff = kWsStatusBytes;
-constexpr size_t kGemmPartialOff = kWsStatusBytes + 8192;
+constexpr size_t kGemmFlags2Off = kWsStatusBytes + 8192;
+constexpr size_t kGemmPartialOff = kGemmFlags2Off + 40960;
 constexpr uint32_t kFlagEmpty = 0x7FA5A5A5u;    // what tman_workspace_init leaves behind
-constexpr size_t partial_bytes_per_cta(int mh) { return (size_t)NUM_EPI_WARPS * mh * (BN / 64) * CHUNK_BYTES; }
+constexpr size_t kPartialBytesPerCta = (size_t)NUM_EPI_WARPS * 2 * (BN / 64) * CHUNK_BYTES;   // 256 KB, whatever MH
 
 struct GemmParams {
     const uint8_t  *packed;
@@ -76,10 +79,12 @@ struct GemmParams {
     const uint16_t *zeros;
     uint32_t       *status;
     uint32_t       *flags;
+    uint32_t       *flags2;
     float          *partial;
     int M, K, N, bits, group;
     int tiles_m, tiles_n;
     int span_tiles;            // the last span_tiles tiles are dealt as equal spans of k-blocks (0: every tile whole)
+    int split_s;               // even split: every tile's k-blocks go to split_s workers (0: off)
     int col_fastest;           // tile number = row tile * tiles_n + column tile (else column tile * tiles_m + row tile)
 };
 
@@ -381,6 +386,11 @@ __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const Co
 // numbers, write their fp32 accumulators to the workspace and raise a flag.  A worker's walk: first
 // the piece that it only contributes (so that it is ready long before it is needed), then its whole
 // tiles, last the piece of the tile that it finishes.
+// Even split (outputs with fewer tiles than half the workers): every tile's k-blocks are cut into S
+// equal pieces for S workers with consecutive numbers.  They finish together; each sends the fp32 chunks
+// that another piece sums into that piece's inbox in the workspace, raises one flag per receiver, then
+// fetches what it was sent and adds it to its own accumulators in piece order: the summing and its
+// traffic are shared by all S workers instead of falling on one.
 struct Segment { int tile, kb0, kb1; bool whole, finishes; };
 
 struct Span {
@@ -393,6 +403,20 @@ struct Span {
         : nu(p.K / (2 * BK)), W(nworkers), w(worker), has_early(false), has_mid(false), has_late(false)
     {
         const long long T = (long long)p.tiles_m * p.tiles_n;
+        if (p.split_s) {
+            // even split: worker w has piece w % S of tile w / S and nothing else
+            full = 0;
+            Ur = 0;
+            next_whole = 0;
+            const int S = p.split_s, piece = worker % S;
+            late.tile = worker / S;
+            late.kb0 = 2 * (int)((long long)nu * piece / S);
+            late.kb1 = 2 * (int)((long long)nu * (piece + 1) / S);
+            late.whole = false;
+            late.finishes = true;
+            has_late = true;
+            return;
+        }
         full = T - p.span_tiles;
         Ur = (long long)p.span_tiles * nu;
         next_whole = worker;
@@ -678,7 +702,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const uint32_t ring_bar = ring0 + 8u * (uint32_t)(ew * PART_RING);
         constexpr size_t WARP_PARTIAL_FLOATS = (size_t)MH * (BN / 64) * (CHUNK_BYTES / 4);
         static_assert(NUM_EPI_WARPS * PART_RING * CHUNK_BYTES <= NSTAGE * A_STAGE_BYTES + NSTAGE * B_STAGE_BYTES, "ring fits in the stages");
-        auto warp_partial = [&](int cta) { return p.partial + ((size_t)cta * NUM_EPI_WARPS + ew) * WARP_PARTIAL_FLOATS; };
+        auto warp_partial = [&](int cta) { return p.partial + (size_t)cta * (kPartialBytesPerCta / 4) + (size_t)ew * WARP_PARTIAL_FLOATS; };
         auto warp_flag = [&](int cta) { return p.flags + (size_t)cta * NUM_EPI_WARPS + ew; };
         uint32_t ti = 0;
         while (ok && span.next(sg)) {
@@ -690,10 +714,129 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const int nq = hv * nch;
             // split tile: the workers before this one that hold the tile's other segments
             int first_w = worker;
-            if (sg.finishes && !sg.whole) first_w = span.owner(sg.tile, 0);
+            if (!p.split_s && sg.finishes && !sg.whole) first_w = span.owner(sg.tile, 0);
             const int ncontrib = worker - first_w;
             if (!mbar_wait(accf, ti & 1u)) { ok = false; break; }
             tcgen05_fence_after();
+            if (p.split_s) {
+                // ---- even split: the S workers of a tile finish together and share the summing -----------
+                // Chunk q of this warp is summed by piece q % S.  A piece first sends the chunks that
+                // others sum (fp32, into their CTA's inbox, slot = (sender, chunk)) and raises one flag
+                // per receiver; then it fetches what the others sent for its own chunks and adds them to
+                // its accumulators in piece order.
+                const int S = p.split_s, me = worker % S, w0 = worker - me;
+                const int CH = (MH * (BN / 64) + S - 1) / S;           // chunks a piece sums, at most
+                auto inbox = [&](int cta, int sender, int slot) {
+                    const int sidx = sender < (cta / NCTA) % S ? sender : sender - 1;
+                    return p.partial + (size_t)cta * (kPartialBytesPerCta / 4) +
+                           ((size_t)(sidx * CH + slot) * NUM_EPI_WARPS + ew) * (CHUNK_BYTES / 4);
+                };
+                auto flag2 = [&](int cta, int sender) { return p.flags2 + ((size_t)cta * NUM_EPI_WARPS + ew) * kMaxSplit + sender; };
+#pragma unroll 1
+                for (int q = 0; q < nq; ++q) {
+                    if (q % S == me) continue;
+                    uint32_t r[32];
+                    tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) +
+                                          (uint32_t)((q / nch) * BN + 32 * epart + 64 * (q % nch)), r);
+                    tcgen05_wait_ld();
+                    float4 *dst = reinterpret_cast<float4 *>(inbox((w0 + q % S) * NCTA + (int)rank, me, q / S)) + lane;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        __stcg(dst + 32 * e, make_float4(__uint_as_float(r[4 * e]), __uint_as_float(r[4 * e + 1]),
+                                                         __uint_as_float(r[4 * e + 2]), __uint_as_float(r[4 * e + 3])));
+                }
+                __threadfence();
+                __syncwarp();
+                if (lane == 0)
+                    for (int o = 0; o < S; ++o)
+                        if (o != me)
+                            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag2((w0 + o) * NCTA + (int)rank, me)), "r"(1u) : "memory");
+                // own chunks: items (own chunk c, other piece o) in that order
+                const int nown = (nq > me) ? (nq - me + S - 1) / S : 0, nitem = nown * (S - 1);
+                auto other = [&](int i) { return i < me ? i : i + 1; };      // i-th other piece
+                auto fetch2 = [&](int jj) {
+                    const int c = jj / (S - 1), o = other(jj % (S - 1));
+                    const uint32_t b = (uint32_t)(jj % PART_RING);
+                    mbar_expect_tx(ring_bar + 8 * b, CHUNK_BYTES);
+                    bulk_load(ring_buf + b * CHUNK_BYTES, inbox((int)blockIdx.x, o, c), CHUNK_BYTES, ring_bar + 8 * b);
+                };
+                if (lane == 0) {
+                    for (int i = 0; i < S - 1 && ok; ++i) {
+                        const uint32_t *f = flag2((int)blockIdx.x, other(i));
+                        uint64_t t0 = 0;
+                        for (uint32_t spin = 0;; ++spin) {
+                            uint32_t fv;
+                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(fv) : "l"(f) : "memory");
+                            if (fv == 1u) break;
+                            if ((spin & 255u) == 255u) {
+                                const uint64_t now = global_timer_ns();
+                                if (t0 == 0) t0 = now;
+                                else if (now - t0 > 1000000000ull) { ok = false; break; }
+                            }
+                        }
+                    }
+                    if (ok) {
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                        for (int jj = 0; jj < PART_RING && jj < nitem; ++jj) fetch2(jj);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                int jj = 0;
+#pragma unroll 1
+                for (int c = 0; c < nown; ++c) {
+                    const int q = me + c * S;
+                    const int h = q / nch, col = 32 * epart + 64 * (q % nch);
+                    const int m0 = rows0 + h * BM + quarter * 32;
+                    uint32_t r[32];
+                    tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * BN + col), r);
+                    tcgen05_wait_ld();
+#pragma unroll 1
+                    for (int i = 0; i < S - 1; ++i, ++jj) {
+                        const uint32_t b = (uint32_t)(jj % PART_RING);
+                        if (!mbar_wait(ring_bar + 8 * b, (uint32_t)(jj / PART_RING) & 1u)) { ok = false; break; }
+                        const uint32_t src = ring_buf + b * CHUNK_BYTES + (uint32_t)lane * 16u;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            float4 a;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w)
+                                         : "r"(src + 512u * e) : "memory");
+                            r[4 * e]     = __float_as_uint(__uint_as_float(r[4 * e]) + a.x);
+                            r[4 * e + 1] = __float_as_uint(__uint_as_float(r[4 * e + 1]) + a.y);
+                            r[4 * e + 2] = __float_as_uint(__uint_as_float(r[4 * e + 2]) + a.z);
+                            r[4 * e + 3] = __float_as_uint(__uint_as_float(r[4 * e + 3]) + a.w);
+                        }
+                        __syncwarp();
+                        if (lane == 0 && jj + PART_RING < nitem) fetch2(jj + PART_RING);
+                    }
+                    if (!ok) break;
+                    uint32_t hv16[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const __half2 hh = __floats2half2_rn(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                        hv16[e] = *reinterpret_cast<const uint32_t *>(&hh);
+                    }
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+#pragma unroll
+                    for (uint32_t cj = 0; cj < 4; ++cj)
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((cj ^ xr) << 4)), "r"(hv16[4 * cj]),
+                                     "r"(hv16[4 * cj + 1]), "r"(hv16[4 * cj + 2]), "r"(hv16[4 * cj + 3]) : "memory");
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) tma_store_2d(&tmap_y, stage, col0 + col, m0);
+                }
+                if (!ok) break;
+                // the accumulators are read; the received flags go back to "empty" for the next launch
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    arrive_lead(acce_lead);
+                    for (int i = 0; i < S - 1; ++i) *flag2((int)blockIdx.x, other(i)) = kFlagEmpty;
+                }
+                ++ti;
+                continue;
+            }
             // issue the fetch of item j = (chunk q, contributor c) into the ring (lane 0)
             auto fetch = [&](int j) {
                 const int q = j / ncontrib, cw = first_w + j % ncontrib;
@@ -849,7 +992,7 @@ inline bool gemm_pair(int M) { return M > BM; }
 // alternative: the widest tiles, whole as far as they go round and the rest in equal spans, whose
 // split tiles cost their workers a partial tile written to and read back from the workspace (an SM
 // writes about 50 GB/s; the more pieces per tile, the more to read back).
-struct GemmPlan { int pair, mh, tiles_m, tiles_n, span_tiles, workers, col_fastest; };
+struct GemmPlan { int pair, mh, tiles_m, tiles_n, span_tiles, workers, col_fastest, split_s; };
 
 GemmPlan plan_gemm(int M, int K, int N, int bits, int sms)
 {
@@ -886,12 +1029,33 @@ GemmPlan plan_gemm(int M, int K, int N, int bits, int sms)
                             (double)((span * nu + workers - 1) / workers) * 2.0 * kb_us(BN) +
                             (span ? (pair ? 24.0 : 16.0) + 3.0 * (double)workers / (double)span : 0.0);
         if (span != 0 && cost < best) {
+            best = cost;
             g.span_tiles = (int)span;
             g.tiles_n = tn_min;
         }
     }
+    g.split_s = 0;
+    {
+        // fewer widest tiles than half the workers: every tile's k-blocks to S workers (even pieces), which
+        // finish together and share the summing
+        const long long t = (long long)g.tiles_m * tn_min;
+        const int nq_warp = g.mh * (BN / 64);           // chunks an epilogue warp holds
+        for (int S = 2; S <= kMaxSplit; ++S) {
+            if (t * S > workers || nu < S) break;
+            if ((S - 1) * ((nq_warp + S - 1) / S) > 8) continue;    // what the pieces send to one CTA must fit its inbox
+            const double cost = (double)((nu + S - 1) / S) * 2.0 * kb_us(BN) + 3.0 +
+                                (pair ? 9.0 + 3.0 * (S - 1) : 8.0 + 1.3 * (S - 1));   // measured exchange times
+            if (cost < best) {
+                best = cost;
+                g.split_s = S;
+                g.span_tiles = 0;
+                g.tiles_n = tn_min;
+            }
+        }
+    }
     const long long tiles = (long long)g.tiles_m * g.tiles_n;
-    if (tiles < workers) {                             // fewer tiles than workers: as many workers as units at most
+    if (g.split_s) workers = tiles * g.split_s;
+    else if (tiles < workers) {                        // fewer tiles than workers: as many workers as units at most
         const long long units = g.span_tiles ? tiles * nu : tiles;
         if (workers > units) workers = units;
     }
@@ -941,18 +1105,20 @@ tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, co
 
 }  // namespace
 
-tman_status mpgemm_plan(int M, int K, int N, int *out6)
+tman_status mpgemm_plan(int M, int K, int N, int *out8)
 {
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
     const GemmPlan g = plan_gemm(M, K, N, 4, sms);
-    out6[0] = g.pair; out6[1] = g.mh; out6[2] = g.tiles_m; out6[3] = g.tiles_n; out6[4] = g.span_tiles ? 0 : 1; out6[5] = g.workers;
+    out8[0] = g.pair; out8[1] = g.mh; out8[2] = g.tiles_m; out8[3] = g.tiles_n; out8[4] = (g.span_tiles || g.split_s) ? 0 : 1; out8[5] = g.workers;
+    out8[6] = g.span_tiles; out8[7] = g.split_s;
     return TMAN_OK;
 }
 
 size_t mpgemm_workspace_bytes(int M, int, int)
 {
-    return kGemmPartialOff + (size_t)kMaxGemmCtas * partial_bytes_per_cta(gemm_mh(M));
+    (void)M;
+    return kGemmPartialOff + (size_t)kMaxGemmCtas * kPartialBytesPerCta;
 }
 
 tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
@@ -1013,11 +1179,13 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.zeros = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
     p.status = reinterpret_cast<uint32_t *>(w8);
     p.flags = reinterpret_cast<uint32_t *>(w8 + kGemmFlagsOff);
+    p.flags2 = reinterpret_cast<uint32_t *>(w8 + kGemmFlags2Off);
     p.partial = reinterpret_cast<float *>(w8 + kGemmPartialOff);
     p.M = M; p.K = K; p.N = N; p.bits = bits; p.group = group;
     p.tiles_m = g.tiles_m;
     p.tiles_n = g.tiles_n;
     p.span_tiles = g.span_tiles;
+    p.split_s = g.split_s;
     p.col_fastest = g.col_fastest;
     if (bits == 2) return launch_bits<2>(tmap_x, tmap_w, tmap_y, p, g, s);
     if (bits == 3) return launch_bits<3>(tmap_x, tmap_w, tmap_y, p, g, s);

@@ -64,16 +64,19 @@ def test_pair_kernel_cases(M, K, N, bits, G):
     check_full(synth.small_case(M, K, N, bits, G, seed=M + K + N + bits, outliers=(bits == 4)))
 
 
-# Long K and few tiles: the last tiles' k-blocks are divided among the workers and summed through
-# the workspace (many pieces per tile).  Pairs of CTAs with two and one row block, a single CTA,
-# ragged M and N, every bit width; compared element by element.
+# Long K and few tiles: every tile's k-blocks go to several workers, which exchange fp32 chunks through
+# the workspace and share the summing.  Pairs of CTAs with two and one row block, a single CTA, ragged
+# M and N, every bit width; compared element by element.
 SPLIT = [(300, 8192, 1024, 4, 128), (520, 8192, 1288, 2, 64), (200, 16384, 520, 3, 128), (100, 24576, 2560, 3, 128)]
+# Slightly fewer tiles than workers (or a few more than a whole round): the last tiles' k-blocks are laid
+# end to end and dealt in equal spans; a tile cut by a span boundary is summed by the worker that ends it.
+SPANS = [(600, 8192, 5120, 4, 128), (1100, 4096, 6400, 2, 64)]
 
 
 @pytest.mark.parametrize("M,K,N,bits,G", SPLIT)
 def test_split_tile_cases(M, K, N, bits, G):
     plan = B.tman_debug_gemm_plan(M, K, N, bits, G)
-    assert plan["whole_tiles"] == 0, plan          # the shape must take the path this test is about
+    assert plan["pieces"] >= 2, plan               # the shape must take the path this test is about
     c = synth.small_case(M, K, N, bits, G, seed=M + K + N + bits)
     check_full(c)
     # the same call again on the same workspace: flags and partial tiles were left ready
@@ -87,6 +90,22 @@ def test_split_tile_cases(M, K, N, bits, G):
         ys.append(y)
     assert B.tman_read_status(ws) == 0
     assert torch.equal(ys[0], ys[1]) and torch.equal(ys[1], ys[2])   # fixed summation order: same bits
+
+
+@pytest.mark.parametrize("M,K,N,bits,G", SPANS)
+def test_span_cases(M, K, N, bits, G):
+    plan = B.tman_debug_gemm_plan(M, K, N, bits, G)
+    assert plan["span_tiles"] > 0, plan            # the shape must take the path this test is about
+    c = synth.small_case(M, K, N, bits, G, seed=M + K + N + bits)
+    y = run_gemm(c)
+    assert bool(torch.isfinite(y).all())
+    rng = np.random.default_rng(M + N)
+    rows = np.unique(np.concatenate([[0, M - 1, 255, 256, 511, 512], rng.integers(0, M, size=26)]))
+    ref = orc.mpgemm_rows(c.x, c.codes, c.scales, c.zeros, c.group, rows)
+    got = H.to_f64(y[torch.from_numpy(rows).cuda()])
+    assert float(np.max(np.abs(got - ref)) / np.max(np.abs(ref))) <= TOL
+    y2 = run_gemm(c)
+    assert torch.equal(y, y2)                       # fixed summation order: same bits
 
 
 def test_integer_case_is_exact():
