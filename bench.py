@@ -422,9 +422,10 @@ def run_ours(args):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
 # profiles/.  mpGEMV: one gate/up-sized launch moved 17.04 MB for 16.78 MB of algorithmic bytes
 # (+1.55 %); traffic grows with the bytes streamed, so the step's mean launch (25.17 MB) is scaled
-# by the same ratio.  mpGEMM: the M=1024, K=4096, N=14336 launch (the larger config-4 shape).
+# by the same ratio.  mpGEMM: none (the kernel has changed since its counters were taken: 41.6 MB for
+# the M=1024, K=4096, N=14336 launch at that time).
 TRAFFIC_BYTES_PER_LAUNCH = 25171968.0 * (17.04 / 16.78)
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = 41.6e6
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
 
 
 def bench_gemm(torch, B, H, synth, peaks):
