@@ -51,7 +51,7 @@ def test_packed_bytes_matches_format_description(lib):
     for K, N, bits, G in [(4096, 4096, 4, 64), (4096, 14336, 2, 64), (14336, 4096, 3, 128), (128, 8, 1, 32)]:
         want = 256 + up(K * N * bits // 8) + up(K // G * N * 2) + up(K // G * (N // 4) * 2)
         assert B.tman_packed_bytes(K, N, bits, G) == want
-    # the survey's figure for config 1: planes + scales (zeros are stored as nibbles)
+    # config 1 (K = N = 4096, 4-bit, group 64): planes + scales (zeros are stored as nibbles)
     assert B.tman_packed_bytes(4096, 4096, 4, 64) == 256 + 8388608 + 524288 + 131072
 
 
