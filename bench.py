@@ -494,7 +494,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--skip-gemm", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--leg", default="headline", choices=["headline", "microbench"],
+                    help="headline: the bench line (default); the others print their own JSON lines")
     args = ap.parse_args()
+    if args.leg != "headline":
+        import bench_legs
+        getattr(bench_legs, args.leg)(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

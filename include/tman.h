@@ -185,6 +185,35 @@ tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_st
  * know which path a shape takes. */
 tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out8 /*host*/);
 
+/* Microbenchmarks behind the decode kernel's design, the counterpart on this GPU of the paper's
+ * instruction study (Sec. 5 "Implementation", Table 1: lookups per instruction x log2(table entries) =
+ * "equivalent multiply-adds" of the 16- and 32-entry lookup instructions) and of its load-path study
+ * (Table 2: DMA, prefetch and vector loads).  One kernel is enqueued per call; nothing of the product
+ * path runs.
+ *   kind 0..6  table-lookup loops, one CTA per SM, arg = threads per CTA (0: 512).  Tables: 0 = 256
+ *              entries fp32, 1 = 256 entries fp16 with a mixed-precision add, 2 = 16 entries fp32 (the
+ *              paper's table shape), 3 = 16 entries held in registers and read with a warp shuffle,
+ *              4 / 5 / 6 = 256 entries that carry 2 / 4 / 8 activation rows in fp16.  results receives one
+ *              u64 per CTA: the clocks its 64 passes over a 16 KB pool of index words took
+ *              (1,048,576 index bytes per CTA: one lookup each for the 256-entry tables, two for the
+ *              16-entry ones).
+ *   kind 10    every CTA streams its share of buffer once with coalesced 16-byte loads (time it with
+ *              events).  kind 11: the same with bulk asynchronous copies of arg bytes into a ring of
+ *              shared-memory stages; a wait that runs out sets results[0] (u32) to TMAN_ERR_TIMEOUT.
+ *   kind 20    clusters of arg CTAs: results[2i], results[2i+1] (u64) = clocks of a cluster barrier, and
+ *              of a store to every peer's shared memory + barrier + read + barrier, for CTA i.
+ *   kind 21    one thread follows a chain of dependent loads through arg bytes of buffer (kept in L2
+ *              when small): results[0] (u64) = clocks per load.
+ * results: device, 256-byte aligned, at least 4096 bytes (its last 256 bytes are scratch); buffer:
+ * device, 256-byte aligned, may be NULL for kinds that do not read it. */
+tman_status tman_debug_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer,
+                                  size_t buffer_bytes, tman_stream_t stream);
+
+/* How many clusters of `cluster` CTAs (threads, dynamic shared memory each) the current device
+ * holds at once (host-side occupancy query, nothing is launched; no counterpart in the paper).  The
+ * decode kernel combines its K-slices inside a cluster, so this number bounds its grid. */
+tman_status tman_debug_cluster_capacity(int threads, int smem_bytes, int cluster, int *out_clusters /*host*/);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,6 +23,7 @@ EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
     "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
+    "tman_debug_microbench", "tman_debug_cluster_capacity",
 ]
 
 _lib = None
@@ -60,6 +61,8 @@ def lib() -> C.CDLL:
         L.tman_debug_indices.argtypes = [vp, i, i, i, i, vp, vp, sz, vp]
         L.tman_debug_luts.argtypes = [vp, i, i, vp, vp]
         L.tman_debug_gemm_plan.argtypes = [i, i, i, i, i, C.POINTER(C.c_int)]
+        L.tman_debug_microbench.argtypes = [i, i, vp, sz, vp, sz, vp]
+        L.tman_debug_cluster_capacity.argtypes = [i, i, i, C.POINTER(C.c_int)]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -172,3 +175,15 @@ def tman_debug_gemm_plan(M, K, N, bits, group) -> dict:
 
 def tman_debug_luts(x, M, K, lut, stream=None) -> None:
     _check(lib().tman_debug_luts(_ptr(x), M, K, _ptr(lut), _stream(stream)), "tman_debug_luts")
+
+
+def tman_debug_microbench(kind, arg, results, buffer=None, stream=None) -> None:
+    _check(lib().tman_debug_microbench(kind, arg, _ptr(results), results.numel() * results.element_size(),
+                                       _ptr(buffer), 0 if buffer is None else buffer.numel() * buffer.element_size(),
+                                       _stream(stream)), "tman_debug_microbench")
+
+
+def tman_debug_cluster_capacity(threads: int, smem_bytes: int, cluster: int) -> int:
+    out = C.c_int(0)
+    _check(lib().tman_debug_cluster_capacity(threads, smem_bytes, cluster, C.byref(out)), "tman_debug_cluster_capacity")
+    return int(out.value)

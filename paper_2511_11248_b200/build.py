@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtman.so")
-SOURCES = ["api.cu", "pack.cu", "mpgemv.cu", "mpgemv_static.cu", "mpgemm.cu"]
+SOURCES = ["api.cu", "pack.cu", "mpgemv.cu", "mpgemv_static.cu", "mpgemm.cu", "microbench.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "--shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,

@@ -182,4 +182,21 @@ tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *
     return mpgemm_plan(M, K, N, out8);
 }
 
+tman_status tman_debug_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer,
+                                  size_t buffer_bytes, tman_stream_t stream)
+{
+    if (!results) return TMAN_ERR_NULL;
+    if (results_bytes < 4096 || (reinterpret_cast<uintptr_t>(results) & 255) || (reinterpret_cast<uintptr_t>(buffer) & 255))
+        return TMAN_ERR_SHAPE;
+    return launch_microbench(kind, arg, results, results_bytes, buffer, buffer_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+tman_status tman_debug_cluster_capacity(int threads, int smem_bytes, int cluster, int *out_clusters)
+{
+    if (!out_clusters) return TMAN_ERR_NULL;
+    if (threads < 32 || threads > 1024 || smem_bytes < 0 || cluster < 1 || cluster > 16) return TMAN_ERR_SHAPE;
+    *out_clusters = cluster_capacity(threads, smem_bytes, cluster);
+    return TMAN_OK;
+}
+
 }  // extern "C"

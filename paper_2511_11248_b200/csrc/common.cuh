@@ -14,7 +14,7 @@ namespace tman {
 // 256-byte header, then bit-plane words, scales, zero-points (each section 256-byte padded).
 struct PackedHeader {
     char     magic[8];      // "TMANB200"
-    uint32_t version;       // 1
+    uint32_t version;       // kVersion
     uint32_t K, N, bits, group, lut_g;
     uint64_t planes_off, scales_off, zeros_off, total_bytes;
 };
@@ -122,5 +122,8 @@ size_t      mpgemm_workspace_bytes(int M, int K, int N);
 tman_status mpgemm_plan(int M, int K, int N, int *out8);
 tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s);
+tman_status launch_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer, size_t buffer_bytes,
+                              cudaStream_t s);
+int         cluster_capacity(int threads, int smem_bytes, int cluster);
 
 }  // namespace tman
