@@ -17,6 +17,7 @@ const char *tman_status_string(int status)
         case TMAN_ERR_BAD_PACKED: return "TMAN_ERR_BAD_PACKED";
         case TMAN_ERR_CUDA: return "TMAN_ERR_CUDA";
         case TMAN_ERR_TIMEOUT: return "TMAN_ERR_TIMEOUT";
+        case TMAN_ERR_LAYOUT: return "TMAN_ERR_LAYOUT";
         default: return "TMAN_ERR_UNKNOWN";
     }
 }
@@ -180,6 +181,24 @@ tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *
     if (st != TMAN_OK) return st;
     if (M < 1) return TMAN_ERR_SHAPE;
     return mpgemm_plan(M, K, N, out8);
+}
+
+tman_status tman_debug_gemv_plan(int count, int M, int K, const int *N, int bits, int group, const int *capacity9, int *out16)
+{
+    if (!N || !out16) return TMAN_ERR_NULL;
+    if (count < 1 || count > 4 || M < 1 || M > 8) return TMAN_ERR_SHAPE;
+    if (bits < 2) return TMAN_ERR_UNSUPPORTED;
+    for (int g = 0; g < count; ++g) {
+        tman_status st = check_format(K, N[g], bits, group);
+        if (st != TMAN_OK) return st;
+    }
+    GemvPlan g;
+    tman_status st = mpgemv_plan(M, K, N, count, bits, group, capacity9, &g);
+    if (st != TMAN_OK) return st;
+    const int v[16] = {g.mt, g.cluster, g.wpc, g.nkt, g.rpp, g.npass, g.ntiles, g.tpc, g.clusters, g.waves, g.stages,
+                       g.smem_bytes, g.tables_bytes, g.park_bytes, g.inbox_bytes, g.cost_clocks};
+    for (int i = 0; i < 16; ++i) out16[i] = v[i];
+    return TMAN_OK;
 }
 
 tman_status tman_debug_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer,

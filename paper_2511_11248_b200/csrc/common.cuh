@@ -113,6 +113,26 @@ tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int
                                  uint32_t *status, cudaStream_t s);
 tman_status launch_debug_luts(const void *x, int M, int K, float *lut, cudaStream_t s);
 size_t      mpgemv_workspace_bytes(int M, int K, int N);
+// How a decode call is cut (see plan_gemv in mpgemv.cu).
+struct GemvPlan {
+    int mt;            // activation rows a table entry carries (1, 2, 4, 8)
+    int cluster;       // CTAs per cluster = K-slices summed on chip
+    int wpc;           // plane words (32 activations) of a K-slice
+    int nkt;           // tile rows of a K-slice
+    int rpp;           // tile rows whose tables are resident at once
+    int npass;         // table builds per CTA
+    int ntiles;        // column tiles of the call
+    int tpc;           // column tiles per cluster
+    int clusters;      // clusters launched
+    int waves;         // rounds of resident clusters
+    int stages;        // ring depth (tiles)
+    int epc;           // output elements a CTA of a cluster finishes
+    int smem_bytes, tables_bytes, park_bytes, inbox_bytes, sums_bytes, sz_bytes;
+    int sz_nbcp, sz_nzw; // staged scales / zero-point words per strip
+    int cost_clocks;   // the model's estimate for the busiest CTA
+};
+GemvPlan    plan_gemv(int M, int K, const int *Ns, int count, int bits, int group, const int *capacity);
+tman_status mpgemv_plan(int M, int K, const int *Ns, int count, int bits, int group, const int *capacity9, GemvPlan *out);
 tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s);
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s);

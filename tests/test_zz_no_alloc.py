@@ -2,7 +2,7 @@
 
 A serving runtime that froze its memory arena, or code running inside another framework's
 callback, has no way to produce the scratch buffer tman_mpgemv wants.  The static variant keeps
-that scratch inside the library (4 MiB per GPU).  It must give what tman_mpgemv gives, call
+that scratch inside the library (4 KiB per GPU).  It must give what tman_mpgemv gives, call
 after call, although every call reuses the same array and finds the previous call's leftovers
 in it.  This file is collected last on purpose: a failure here cannot hide another test's.
 """
@@ -54,13 +54,8 @@ def test_same_problem_twice_gives_the_same_answer():
         assert float(np.max(np.abs(got - want)) / np.max(np.abs(want))) <= TOL
 
 
-def test_shape_beyond_the_fixed_array_is_refused():
-    # scratch for K = 18944, N = 18944 is far above 4 MiB: refused on the host, nothing enqueued
-    K, N, bits, G = 18944, 18944, 2, 128
-    assert B.tman_workspace_bytes(B.OP_GEMV, 1, K, N, bits, G) > (4 << 20)
-    packed = torch.empty(B.tman_packed_bytes(K, N, bits, G), dtype=torch.uint8, device="cuda")
-    x = torch.zeros((1, K), dtype=torch.float16, device="cuda")
-    y = torch.zeros((1, N), dtype=torch.float16, device="cuda")
-    with pytest.raises(B.TmanError) as e:
-        B.tman_mpgemv_static(packed, x, y, 1, K, N, bits, G)
-    assert e.value.status == 4   # TMAN_ERR_BUFFER_TOO_SMALL
+def test_no_legal_shape_outgrows_the_fixed_array():
+    # the array is 4 KiB; the decode path's global scratch is its status block, whatever the shape, so the
+    # size check of the entry point never refuses a legal decode shape
+    for M, K, N, bits, G in [(8, 18944, 18944, 2, 128), (1, 4096, 152064, 4, 32), (8, 128, 8, 4, 128)]:
+        assert B.tman_workspace_bytes(B.OP_GEMV, M, K, N, bits, G) <= 4096
