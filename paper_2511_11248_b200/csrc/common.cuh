@@ -127,8 +127,8 @@ struct GemvPlan {
     int waves;         // rounds of resident clusters
     int stages;        // ring depth (tiles)
     int epc;           // output elements a CTA of a cluster finishes
-    int smem_bytes, tables_bytes, park_bytes, inbox_bytes, sums_bytes, sz_bytes;
-    int sz_nbcp, sz_nzw; // staged scales / zero-point words per strip
+    int smem_bytes, tables_bytes, park_bytes, inbox_bytes, sums_bytes;
+    int sz_tma, nbt, zw, stage_bytes;   // scales and zero-points copied with the tile (1/0), blocks per tile row, zero-point row, stage size
     int cost_clocks;   // the model's estimate for the busiest CTA
 };
 GemvPlan    plan_gemv(int M, int K, const int *Ns, int count, int bits, int group, const int *capacity);

@@ -91,7 +91,8 @@ struct Cfg {
     static constexpr int PARK_TILE_BYTES = 8 * 32 * VPL * 4;     // parked sums of a tile's eight items
 };
 
-struct TMaps { CUtensorMap m[kGemvMaxGroup]; };
+// bit-plane words (3-D), scales (2-D, 32-bit pairs of fp16) and zero-points (2-D, 16-bit) of every matrix
+struct TMaps { CUtensorMap m[kGemvMaxGroup]; CUtensorMap sc[kGemvMaxGroup]; CUtensorMap z[kGemvMaxGroup]; };
 
 struct GemvParams {
     const uint8_t  *packed[kGemvMaxGroup];
@@ -115,8 +116,11 @@ struct GemvParams {
     int npass;
     int stages;                 // ring depth
     int epc;                    // output elements (column x row) each CTA of a cluster finishes
-    uint32_t ring_off, park_off, inbox_off, sums_off, sz_off, bar_off;   // shared-memory layout (bytes from the dynamic base)
-    int sz_nbcp, sz_nzw;        // staged scales / zero-point words per strip (row lengths of the staging area)
+    uint32_t ring_off, park_off, inbox_off, sums_off, bar_off;   // shared-memory layout (bytes from the dynamic base)
+    int sz_tma;                 // 1: a tile's scales and zero-points are copied into its stage (needs nblk % 8 == 0)
+    int nbt;                    // quantization blocks of a tile row
+    int zw;                     // zero-point entries per strip in a stage (a copy starts at a multiple of 8 entries)
+    int stage_bytes;            // bit-plane words, then scales, then zero-points
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -168,6 +172,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tma
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tmap, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
@@ -350,8 +360,13 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     cluster_arrive_relaxed();
     if (tid == 0) {
-        for (int g = 0; g < p.count; ++g)
+        for (int g = 0; g < p.count; ++g) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.m[g])) : "memory");
+            if (p.sz_tma) {
+                asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.sc[g])) : "memory");
+                asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&maps.z[g])) : "memory");
+            }
+        }
         for (int i = 0; i < p.stages; ++i) {
             mbar_init(full0 + 8u * i, 1);
             mbar_init(empty0 + 8u * i, 8);
@@ -388,34 +403,6 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
         meta[tid] = tm;
     }
     __syncthreads();
-
-    // Ask for the scales and zero-points of this CTA's share to be brought into L2 (a hint: nothing is
-    // read into the SM, so it is safe whatever the previous kernel of the stream still writes).
-    {
-        const int blk0 = (cta_w0 * 32) / p.group, blk1 = (cta_w1 * 32 + p.group - 1) / p.group;
-        const int sc_lines = ((blk1 - blk0) * 8 + 127) / 128 + 1, z_lines = ((blk1 - blk0) * 2 + 127) / 128 + 1;
-        const int per_strip = sc_lines + z_lines;
-        const int nwork = ntl * C_::TS * per_strip;
-        for (int w = tid; w < nwork; w += kGemvThreads) {
-            const int si = w / per_strip, li = w - si * per_strip;
-            const int T = tile_lo + si / C_::TS;
-            int m = 0;
-#pragma unroll
-            for (int t = 1; t < kGemvMaxGroup; ++t) m += (t < p.count && T >= p.tile0[t]) ? 1 : 0;
-            const int nb = (T - p.tile0[m]) * C_::TS + si % C_::TS;
-            if (nb < (p.Ng[m] >> 2)) {
-                const uint8_t *a;
-                if (li < sc_lines) {
-                    a = reinterpret_cast<const uint8_t *>(p.scales[m]) + ((size_t)nb * p.nblk + blk0) * 8 + (size_t)li * 128;
-                    if (li * 128 >= (blk1 - blk0) * 8 + 127) a = nullptr;
-                } else {
-                    a = reinterpret_cast<const uint8_t *>(p.zeros[m]) + ((size_t)nb * p.nblk + blk0) * 2 + (size_t)(li - sc_lines) * 128;
-                    if ((li - sc_lines) * 128 >= (blk1 - blk0) * 2 + 127) a = nullptr;
-                }
-                if (a) asm volatile("prefetch.global.L2 [%0];" ::"l"(a));
-            }
-        }
-    }
 
     // Nothing of the caller's memory is read into the SM before this point: everything below may depend
     // on the previous kernel of the stream.
@@ -461,22 +448,29 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
         }
         if (ok && round > 0) ok = mbar_wait(empty0 + 8u * st, (round - 1) & 1u, flags);
         if (ok) ok = in_range(st < (uint32_t)p.stages && 2 * iq + gq < ntl && rq < rows_q && tm.m >= 0 && tm.m < p.count &&
-                              p.ring_off + (st + 1) * C_::TILE_BYTES <= p.park_off, 1);
+                              p.ring_off + (st + 1) * (uint32_t)p.stage_bytes <= p.park_off, 1);
         if (!ok) {
             issue_ok = false;
             if (!flags[1] && !flags[0]) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
             flags[0] = 1;
             return;
         }
-        mbar_expect_tx(full0 + 8u * st, C_::TILE_BYTES);
-        tma_load_3d(smem_u32(smem + p.ring_off) + st * C_::TILE_BYTES, &maps.m[tm.m],
-                    (cta_w0 + (row0 + rq) * C_::TW) * 4, 0, tm.strip0, full0 + 8u * st);
+        const uint32_t dst = smem_u32(smem + p.ring_off) + st * (uint32_t)p.stage_bytes;
+        const int w_tile = cta_w0 + (row0 + rq) * C_::TW;                 // first plane word of the tile
+        const uint32_t sc_bytes = (uint32_t)(C_::TS * p.nbt * 8), z_bytes = (uint32_t)(C_::TS * p.zw * 2);
+        mbar_expect_tx(full0 + 8u * st, C_::TILE_BYTES + (p.sz_tma ? sc_bytes + z_bytes : 0u));
+        tma_load_3d(dst, &maps.m[tm.m], w_tile * 4, 0, tm.strip0, full0 + 8u * st);
+        if (p.sz_tma) {
+            const int blk = w_tile >> p.wshift;                            // first block of the tile row
+            tma_load_2d(dst + C_::TILE_BYTES, &maps.sc[tm.m], blk * 2, tm.strip0, full0 + 8u * st);
+            tma_load_2d(dst + C_::TILE_BYTES + sc_bytes, &maps.z[tm.m], blk & ~7, tm.strip0, full0 + 8u * st);
+        }
         __threadfence_block();
         flags[2] = q + 1;
     };
     // every warp: issue my next tile once it falls inside the window that starts at tile `first_in_use`
-    auto issue_due = [&](uint32_t first_in_use) {
-        if (my_q < total_tiles && my_q < first_in_use + ahead_tiles && issue_ok) {
+    auto issue_due = [&](uint32_t first_in_use, uint32_t ahead) {
+        if (my_q < total_tiles && my_q < first_in_use + ahead && issue_ok) {
             if (lane == 0) issue_tile(my_q);
             my_q += kGemvWarps;
         }
@@ -524,32 +518,32 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
         const int row0 = pass * p.rpp, rows = min(p.rpp, p.nkt - row0);
         if (pass > 0) __syncthreads();              // everyone is done with the previous pass's tables
 
-        // ---- scales and zero-points of this pass: copied asynchronously (cp.async) into shared memory while
-        // the tables are built, so that the lookup loop issues no global load of its own (small loads would
-        // queue behind the tile copies).  Scales: 8 bytes per (strip, block); zero-points: the 4-byte words
-        // that hold the 2-byte entries of the strip's blocks (the entry of block b sits at index
-        // e0 + b - blk_a of the strip's words, e0 = parity of the strip's first entry).
-        const int w_a = cta_w0 + row0 * C_::TW, w_b = min(cta_w0 + (row0 + rows) * C_::TW, p.words_total);
-        const int blk_a = min(w_a >> p.wshift, p.nblk - 1);
-        const int blk_b = min(((max(w_b, w_a + 1) - 1) >> p.wshift) + 1, p.nblk);
-        const int nbc = max(blk_b - blk_a, 1);
-        auto stage_sz = [&]() {      // a warp takes a strip at a time, its lanes the strip's blocks
-            uint2 *sc_st = reinterpret_cast<uint2 *>(smem + p.sz_off);
-            uint32_t *z_st = reinterpret_cast<uint32_t *>(smem + p.sz_off + (size_t)p.tpc * C_::TS * p.sz_nbcp * 8);
-            for (int st_ = warp; st_ < ntl * C_::TS; st_ += kGemvWarps) {
-                const TileMeta tm = meta[st_ / C_::TS];
-                const int nb = min(st_ % C_::TS, tm.nleft - 1);
-                const size_t e = (size_t)nb * p.nblk + blk_a;      // the strip's first entry of this pass
-                const int odd = (int)(((reinterpret_cast<uintptr_t>(tm.z) >> 1) + e) & 1);
-                for (int k = lane; k < nbc; k += 32)
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;"
-                                 ::"r"(smem_u32(sc_st + (size_t)st_ * p.sz_nbcp + k)), "l"(tm.sc + (e + k) * 2) : "memory");
-                for (int k = lane; 2 * k < odd + nbc; k += 32)     // the words that hold an entry of the pass
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
-                                 ::"r"(smem_u32(z_st + (size_t)st_ * p.sz_nzw + k)), "l"(tm.z + e - odd + 2 * k) : "memory");
+        // Scales and zero-points: with the tile in its stage (see issue_tile), or, where the block count
+        // rules that out, fetched by every lane one step ahead of their use.
+        struct ScaleZero { uint32_t sc0, sc1, z0, z1; };
+        auto fetch_sz = [&](int i, int r) {
+            ScaleZero v = {0u, 0u, 0u, 0u};
+            const int tl = 2 * i + grp;
+            if (!p.sz_tma && tl < ntl && r < rows) {
+                const TileMeta tm = meta[tl];
+                const int nb = min(js * 8 + s, tm.nleft - 1);
+                const uint32_t *psc = tm.sc + (size_t)nb * p.nblk * 2 + hl;
+                const uint16_t *pz = tm.z + (size_t)nb * p.nblk;
+                const int gw_pair = cta_w0 + (row0 + r) * C_::TW + jk * 8 + 2 * pair_in_part;
+                const int b0 = min(gw_pair >> p.wshift, p.nblk - 1);
+                v.sc0 = __ldg(psc + 2 * b0);
+                v.z0 = __ldg(pz + b0);
+                v.sc1 = v.sc0;
+                v.z1 = v.z0;
+                if (per_word) {
+                    const int b1 = min((gw_pair + 1) >> p.wshift, p.nblk - 1);
+                    v.sc1 = __ldg(psc + 2 * b1);
+                    v.z1 = __ldg(pz + b1);
+                }
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
+            return v;
         };
+        ScaleZero ahead_sz = fetch_sz(0, 0);
         TMAN_CLK_DECL;
 
         // ---- phase A: tables of this pass (paper Sec. 2.2; one table per 8 activations, 256 entries,
@@ -606,9 +600,9 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
             }
         }
         TMAN_CLK(8);
-        stage_sz();
-        __syncthreads();
-        if (pass == 0) issue_due(0u);
+        // the first tiles are asked for while the activations are on their way (a short window: the issuing
+        // thread is held while the copy engine's queue is full, and the tables wait for every warp)
+        if (pass == 0) issue_due(0u, min(ahead_tiles, 4u));
         TMAN_CLK(9);
 #pragma unroll
         for (int v = 0; v < 2; ++v) {
@@ -665,7 +659,6 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
             sums[tid] = sacc;              // index (r * TW + word slot) * MT + row
         }
         TMAN_CLK(10);
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncthreads();
         TMAN_CLK(11);
         TMAN_STAMP(3);
@@ -679,37 +672,13 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
             float yv[C_::NV];
 #pragma unroll
             for (int e = 0; e < C_::NV; ++e) yv[e] = 0.f;
-            int zpar = 0;          // whether the lane's first zero-point entry is the upper half of its staged word
-            if (have) {
-                const TileMeta tm = meta[tl];
-                const int nb = min(js * 8 + s, tm.nleft - 1);
-                zpar = (int)(((reinterpret_cast<uintptr_t>(tm.z) >> 1) + (size_t)nb * p.nblk + blk_a) & 1);
-            }
             for (int r = 0; r < rows; ++r) {
                 const uint32_t seq_pair = seq_base + (uint32_t)((2 * i) * rows + r * cnt_i);
-                issue_due(seq_pair);
+                issue_due(seq_pair, ahead_tiles);
                 if (!have) continue;
                 TMAN_CLK(0);
-                uint32_t sc0, sc1, z0, z1;
-                {
-                    const int gw_pair = cta_w0 + (row0 + r) * C_::TW + jk * 8 + 2 * pair_in_part;
-                    const int b0 = min(gw_pair >> p.wshift, p.nblk - 1) - blk_a;
-                    const int sl = tl * C_::TS + js * 8 + s;
-                    const uint32_t *scp = reinterpret_cast<const uint32_t *>(smem + p.sz_off) + ((size_t)sl * p.sz_nbcp + b0) * 2 + hl;
-                    const uint16_t *zp = reinterpret_cast<const uint16_t *>(smem + p.sz_off + (size_t)p.tpc * C_::TS * p.sz_nbcp * 8) +
-                                         (size_t)sl * p.sz_nzw * 2 + zpar + b0;
-                    if (!in_range(b0 >= 0 && b0 + (per_word ? 1 : 0) < p.sz_nbcp && sl >= 0 && sl < p.tpc * C_::TS &&
-                                  2 * (zpar + b0 + 1) <= 4 * p.sz_nzw, 3)) { alive = false; break; }
-                    sc0 = scp[0];
-                    z0 = (uint32_t)zp[0] >> (8 * hl);
-                    sc1 = sc0;
-                    z1 = z0;
-                    if (per_word) {
-                        const int b1 = min((gw_pair + 1) >> p.wshift, p.nblk - 1) - blk_a - b0;
-                        sc1 = scp[2 * b1];
-                        z1 = (uint32_t)zp[b1] >> (8 * hl);
-                    }
-                }
+                const ScaleZero now_sz = ahead_sz;
+                if (!p.sz_tma) ahead_sz = (r + 1 < rows) ? fetch_sz(i, r + 1) : fetch_sz(i + 1, 0);
                 TMAN_CLK(1);
                 const uint32_t seq = seq_pair + (uint32_t)grp;
                 const uint32_t round = (uint32_t)(((float)seq + 0.5f) * inv_stages), st = seq - round * (uint32_t)p.stages;
@@ -723,7 +692,28 @@ mpgemv_kernel(const __grid_constant__ TMaps maps, const __grid_constant__ GemvPa
                 }
                 TMAN_CLK(2);
                 if (i == 0 && r == 0 && pass == 0) TMAN_STAMP(8);          // latest first-tile arrival over the warps
-                const uint32_t tile_addr = ring + st * C_::TILE_BYTES + lane_off;
+                const uint32_t stage_addr = ring + st * (uint32_t)p.stage_bytes;
+                const uint32_t tile_addr = stage_addr + lane_off;
+                uint32_t sc0 = now_sz.sc0, sc1 = now_sz.sc1, z0 = now_sz.z0, z1 = now_sz.z1;
+                if (p.sz_tma) {
+                    // the tile's scales [strip][block] (8 bytes) and zero-points [strip][zw] (2 bytes) behind its words
+                    const int w_tile = cta_w0 + (row0 + r) * C_::TW;
+                    const int blk_tile = w_tile >> p.wshift;
+                    const int b0 = (w_tile + jk * 8 + 2 * pair_in_part) >> p.wshift;
+                    const uint32_t sc_a = stage_addr + C_::TILE_BYTES + (uint32_t)(((js * 8 + s) * p.nbt + (b0 - blk_tile)) * 8 + hl * 4);
+                    const uint32_t z_a = stage_addr + C_::TILE_BYTES + (uint32_t)(C_::TS * p.nbt * 8) +
+                                         (uint32_t)(((js * 8 + s) * p.zw + (b0 - (blk_tile & ~7))) * 2);
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc0) : "r"(sc_a));
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(z0) : "r"(z_a));
+                    sc1 = sc0;
+                    z1 = z0;
+                    if (per_word) {
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc1) : "r"(sc_a + 8u));
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(z1) : "r"(z_a + 2u));
+                    }
+                }
+                z0 >>= 8 * hl;
+                z1 >>= 8 * hl;
                 const float *srow = sums + (size_t)(r * C_::TW + jk * 8 + 2 * pair_in_part) * MT;
                 float S0[MT], S1[MT];
 #pragma unroll
@@ -977,10 +967,12 @@ GemvPlan plan_gemv(int M, int K, const int *Ns, int count, int bits, int group, 
         const int tables = rpp * v.row_bytes;
         const int sums = up256(rpp * v.tw * mt * 4);
         const int fixed = tables + sums + 2 * kGemvMaxStages * 8 + 64 + kGemvMaxTilesPerCluster * 32;
-        // staged scales and zero-points of a pass: per strip (blocks of the pass + 1) * 8 bytes (one spare
-        // entry keeps the strips' rows off each other's banks) and (blocks / 2 + 2) * 4 bytes
-        const int nbc_max = (rpp * v.tw * 32) / group + 1;
-        const int sz_nbcp = nbc_max + 1, sz_nzw = nbc_max / 2 + 2;
+        // a stage holds a tile's bit-plane words and, where the copy engine can address them (rows of the
+        // zero-point array a multiple of 16 bytes apart), its scales and zero-points
+        // (a zero-point copy starts at a multiple of 8 entries = 16 bytes, so its rows are up to 8 entries wider)
+        const int nbt = (v.tw * 32) / group, zw = nbt >= 8 ? nbt + 8 : 8;
+        const int sz_tma = ((K / group) % 8 == 0) ? 1 : 0;
+        const int stage_bytes = (v.tile_bytes + (sz_tma ? v.ts * (nbt * 8 + zw * 2) : 0) + 127) / 128 * 128;
         // the most tiles per cluster whose parked sums and inbox still leave room for the ring
         int even = (ntiles + capacity[C] - 1) / capacity[C];
         if (even > kGemvMaxTilesPerCluster) even = kGemvMaxTilesPerCluster;
@@ -989,10 +981,9 @@ GemvPlan plan_gemv(int M, int K, const int *Ns, int count, int bits, int group, 
             const int waves = (ncl + capacity[C] - 1) / capacity[C];
             const int epc = (tpc * v.tc * mt + C - 1) / C;
             const int park = up256(tpc * v.park_tile_bytes);
-            const int sz = up256(tpc * v.ts * (sz_nbcp * 8 + sz_nzw * 4));
             const int inbox = up256(C * epc * 4);
             const int tiles_cta = tpc * nkt;                  // tiles a CTA streams
-            int stages = (kGemvSmemLimit - fixed - park - inbox - sz) / v.tile_bytes;
+            int stages = (kGemvSmemLimit - fixed - park - inbox) / stage_bytes;
             if (stages > kGemvMaxStages) stages = kGemvMaxStages;
             if (stages > tiles_cta) stages = tiles_cta;
             if (stages < (tiles_cta < 2 ? tiles_cta : 2)) {
@@ -1005,7 +996,7 @@ GemvPlan plan_gemv(int M, int K, const int *Ns, int count, int bits, int group, 
             const double pairs = (tpc + 1) / 2;               // two tiles are worked on at a time
             const double unit_wf = 2.0 * bits * (2.0 + 8.0 * wf_lookup);     // one warp, one tile row
             const double lookups = pairs * kGemvWarps * nkt * unit_wf / pipe_use;
-            const double stream = (double)tiles_cta * v.tile_bytes / 22.0;   // HBM share of an SM: ~22 bytes per clock
+            const double stream = (double)tiles_cta * stage_bytes / 22.0;    // HBM share of an SM: ~22 bytes per clock
             const double build = (double)npass * (tables / 128.0 + 500.0);
             const double exchange = 700.0 + 90.0 * C;
             const double cost = waves * (build + (lookups > stream ? lookups : stream) + exchange + 1200.0);
@@ -1014,8 +1005,8 @@ GemvPlan plan_gemv(int M, int K, const int *Ns, int count, int bits, int group, 
                 best.mt = mt; best.cluster = C; best.wpc = wpc; best.nkt = nkt; best.rpp = rpp; best.npass = npass;
                 best.ntiles = ntiles; best.tpc = tpc; best.clusters = ncl; best.waves = waves; best.stages = stages;
                 best.epc = epc; best.tables_bytes = tables; best.park_bytes = park; best.inbox_bytes = inbox;
-                best.sums_bytes = sums; best.sz_bytes = sz; best.sz_nbcp = sz_nbcp; best.sz_nzw = sz_nzw;
-                best.smem_bytes = fixed + park + inbox + sz + stages * v.tile_bytes;
+                best.sums_bytes = sums; best.sz_tma = sz_tma; best.nbt = nbt; best.zw = zw; best.stage_bytes = stage_bytes;
+                best.smem_bytes = fixed + park + inbox + stages * stage_bytes;
                 best.cost_clocks = (int)cost;
             }
             if (waves == 1) break;                            // fewer tiles per cluster only cost more from here
@@ -1035,13 +1026,14 @@ tman_status launch_variant(const TMaps &maps, GemvParams &p, const GemvPlan &g, 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvSmemLimit) != cudaSuccess)
         return TMAN_ERR_CUDA;
     p.ring_off = (uint32_t)g.tables_bytes;
-    p.park_off = p.ring_off + (uint32_t)(g.stages * C_::TILE_BYTES);
+    p.park_off = p.ring_off + (uint32_t)(g.stages * g.stage_bytes);
     p.inbox_off = p.park_off + (uint32_t)g.park_bytes;
     p.sums_off = p.inbox_off + (uint32_t)g.inbox_bytes;
-    p.sz_off = p.sums_off + (uint32_t)g.sums_bytes;
-    p.bar_off = p.sz_off + (uint32_t)g.sz_bytes;
-    p.sz_nbcp = g.sz_nbcp;
-    p.sz_nzw = g.sz_nzw;
+    p.bar_off = p.sums_off + (uint32_t)g.sums_bytes;
+    p.sz_tma = g.sz_tma;
+    p.nbt = g.nbt;
+    p.zw = g.zw;
+    p.stage_bytes = g.stage_bytes;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(g.clusters * g.cluster));
     cfg.blockDim = dim3(kGemvThreads);
@@ -1148,6 +1140,27 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
                 wbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return TMAN_ERR_CUDA;
+        if (g.sz_tma) {
+            // scales: (pairs of fp16 of a strip's blocks, strip); zero-points: (16-bit entry of a block, strip)
+            const cuuint64_t nblk = (cuuint64_t)(K / group);
+            const cuuint64_t sdims[2] = {nblk * 2, (cuuint64_t)(Ns[mm] / 4)};
+            const cuuint64_t sstrides[1] = {nblk * 8};
+            const cuuint32_t sbox[2] = {(cuuint32_t)(g.nbt * 2), (cuuint32_t)v.ts};
+            if (enc(&maps.sc[m], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint8_t *>(pk + L.scales_off), sdims, sstrides,
+                    sbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return TMAN_ERR_CUDA;
+            const cuuint64_t zdims[2] = {nblk, (cuuint64_t)(Ns[mm] / 4)};
+            const cuuint64_t zstrides[1] = {nblk * 2};
+            const cuuint32_t zbox[2] = {(cuuint32_t)g.zw, (cuuint32_t)v.ts};
+            if (enc(&maps.z[m], CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint8_t *>(pk + L.zeros_off), zdims, zstrides,
+                    zbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return TMAN_ERR_CUDA;
+        } else {
+            maps.sc[m] = maps.m[m];
+            maps.z[m] = maps.m[m];
+        }
     }
     p.tile0[kGemvMaxGroup] = tiles;
     for (int m = count; m < kGemvMaxGroup; ++m) p.tile0[m] = tiles;
@@ -1160,8 +1173,8 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
     p.ntiles = g.ntiles;
     p.tpc = g.tpc; p.wpc = g.wpc; p.nkt = g.nkt; p.rpp = g.rpp; p.npass = g.npass;
     p.stages = g.stages; p.epc = g.epc;
-    p.ring_off = p.park_off = p.inbox_off = p.sums_off = p.sz_off = p.bar_off = 0;
-    p.sz_nbcp = p.sz_nzw = 0;
+    p.ring_off = p.park_off = p.inbox_off = p.sums_off = p.bar_off = 0;
+    p.sz_tma = p.nbt = p.zw = p.stage_bytes = 0;
     switch (bits * 10 + mt_index(g.mt)) {
         case 20: return launch_variant<2, 1>(maps, p, g, s);
         case 21: return launch_variant<2, 2>(maps, p, g, s);
