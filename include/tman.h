@@ -66,7 +66,7 @@ tman_status tman_packed_bytes(int K, int N, int bits, int group, size_t *out_byt
 tman_status tman_workspace_bytes(int op, int M, int K, int N, int bits, int group,
                                  size_t *out_bytes /*host*/);
 
-/* Prepare a workspace: status word zero, the flag area of the prefill path marked empty.  After a call
+/* Prepare a workspace: status word zero, partial-sum area marked "no sum pending".  After a call
  * reported TMAN_ERR_TIMEOUT the workspace must be prepared again. */
 tman_status tman_workspace_init(void *workspace, size_t ws_bytes, tman_stream_t stream);
 
@@ -104,7 +104,17 @@ tman_status tman_unpack_weights(const void *packed, size_t packed_bytes,
  * packed_bytes is the size of the caller's packed allocation; it must be at least
  * tman_packed_bytes(K, N, bits, group) (else TMAN_ERR_BUFFER_TOO_SMALL).  With that guarantee the
  * kernels may start streaming weights before the header check has completed; a header that does
- * not match the arguments still leaves y untouched and sets the status word. */
+ * not match the arguments still leaves y untouched and sets the status word.
+ *
+ * Stream order of the packed buffer.  The decode calls are launched so that they may begin while
+ * the kernel before them on `stream` is still draining (programmatic dependent launch), and they
+ * read the packed buffer in that window.  What is safe without further care: a packed buffer
+ * written by tman_pack_weights on the same stream (the library puts the next decode call in plain
+ * stream order), by a memory copy, or by any kernel that does not signal early completion.  What
+ * is not: a kernel of the caller's own that calls cudaTriggerProgrammaticLaunchCompletion (PTX
+ * griddepcontrol.launch_dependents) and then writes the packed buffer, directly followed by a decode
+ * call on the same stream -- put an event or another kernel between them.  Activations and the
+ * workspace have no such rule: they are read only after the predecessor has completed. */
 
 /* Decode (paper Sec. 2.2 "Bit-serial table lookup", Fig. 2; Sec. 4.3): activation tables are
  * built in shared memory, packed bit-plane bytes index them, partial sums are
@@ -147,13 +157,12 @@ tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f
  * For callers that may not allocate device memory when they need a matmul -- a runtime that fixed
  * its arena at start-up, code running inside another framework's callback, a region where the
  * allocator is locked -- and so cannot produce the workspace tman_mpgemv asks for.  The scratch
- * is a fixed 4 KiB array inside the library image; every GPU that loads the library holds it
+ * is a fixed 4 MiB array inside the library image; every GPU that loads the library holds it
  * until the process exits, and this call allocates and frees nothing.
  *
  *   - Same result as tman_mpgemv for the same arguments (same kernels, same summation order).
- *   - A shape whose scratch, tman_workspace_bytes(0, M, K, N, bits, group), exceeds 4 KiB is
- *     refused with TMAN_ERR_BUFFER_TOO_SMALL before anything is enqueued (the decode path keeps only its
- *     status block in global memory, so no legal shape is refused today).
+ *   - A shape whose scratch, tman_workspace_bytes(0, M, K, N, bits, group), exceeds 4 MiB is
+ *     refused with TMAN_ERR_BUFFER_TOO_SMALL before anything is enqueued.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents: each
@@ -186,18 +195,6 @@ tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_st
  * spans (0: none); pieces every tile's k-blocks are split into (0: not split).  Tests use it to
  * know which path a shape takes. */
 tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out8 /*host*/);
-
-/* How tman_mpgemv / tman_mpgemv_grouped would cut a call (host-side decision, nothing is launched): the
- * counterpart of the paper's constraint-driven tiling search (Sec. 4.1, Eq. 1-4 and its heuristics) with
- * this GPU's limits in place of the NPU's: shared memory for tables, ring, parked sums and inbox; how many
- * clusters of a size run at once.  capacity9 (host, may be NULL): clusters of 0..8 CTAs the device holds at
- * once, index = cluster size; NULL asks the current device.  out16 (host) receives: activation rows per
- * table entry; CTAs per cluster (K-slices summed on chip); plane words (32 activations) per K-slice; tile
- * rows of a K-slice; tile rows whose tables are resident at once; table builds per CTA; column tiles of
- * the call; column tiles per cluster; clusters launched; waves of resident clusters; ring depth in tiles;
- * shared memory bytes in total, of the tables, of the parked sums, of the inbox; the cost model's clocks. */
-tman_status tman_debug_gemv_plan(int count, int M, int K, const int *N /*host*/, int bits, int group,
-                                 const int *capacity9 /*host*/, int *out16 /*host*/);
 
 /* Microbenchmarks behind the decode kernel's design, the counterpart on this GPU of the paper's
  * instruction study (Sec. 5 "Implementation", Table 1: lookups per instruction x log2(table entries) =

@@ -23,7 +23,7 @@ EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
     "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
-    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemv_plan",
+    "tman_debug_microbench", "tman_debug_cluster_capacity",
 ]
 
 _lib = None
@@ -61,7 +61,6 @@ def lib() -> C.CDLL:
         L.tman_debug_indices.argtypes = [vp, i, i, i, i, vp, vp, sz, vp]
         L.tman_debug_luts.argtypes = [vp, i, i, vp, vp]
         L.tman_debug_gemm_plan.argtypes = [i, i, i, i, i, C.POINTER(C.c_int)]
-        L.tman_debug_gemv_plan.argtypes = [i, i, i, C.POINTER(i), i, i, C.POINTER(i), C.POINTER(i)]
         L.tman_debug_microbench.argtypes = [i, i, vp, sz, vp, sz, vp]
         L.tman_debug_cluster_capacity.argtypes = [i, i, i, C.POINTER(C.c_int)]
         for name in EXPORTS[2:]:
@@ -189,19 +188,3 @@ def tman_debug_cluster_capacity(threads: int, smem_bytes: int, cluster: int) -> 
     _check(lib().tman_debug_cluster_capacity(threads, smem_bytes, cluster, C.byref(out)), "tman_debug_cluster_capacity")
     return int(out.value)
 
-
-GEMV_PLAN_FIELDS = ("rows_per_entry", "cluster", "words_per_slice", "tile_rows", "rows_resident", "passes", "tiles",
-                    "tiles_per_cluster", "clusters", "waves", "stages", "smem_bytes", "tables_bytes", "park_bytes",
-                    "inbox_bytes", "cost_clocks")
-
-
-def tman_debug_gemv_plan(M, K, N_list, bits, group, capacity=None) -> dict:
-    """How a decode call would be cut; capacity = resident clusters by cluster size (9 entries) or None."""
-    if isinstance(N_list, int):
-        N_list = [N_list]
-    n = len(N_list)
-    ns = (C.c_int * n)(*[int(v) for v in N_list])
-    cap = None if capacity is None else (C.c_int * 9)(*[int(v) for v in capacity])
-    out = (C.c_int * 16)()
-    _check(lib().tman_debug_gemv_plan(n, M, K, ns, bits, group, cap, out), "tman_debug_gemv_plan")
-    return dict(zip(GEMV_PLAN_FIELDS, list(out)))

@@ -183,24 +183,6 @@ tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *
     return mpgemm_plan(M, K, N, out8);
 }
 
-tman_status tman_debug_gemv_plan(int count, int M, int K, const int *N, int bits, int group, const int *capacity9, int *out16)
-{
-    if (!N || !out16) return TMAN_ERR_NULL;
-    if (count < 1 || count > 4 || M < 1 || M > 8) return TMAN_ERR_SHAPE;
-    if (bits < 2) return TMAN_ERR_UNSUPPORTED;
-    for (int g = 0; g < count; ++g) {
-        tman_status st = check_format(K, N[g], bits, group);
-        if (st != TMAN_OK) return st;
-    }
-    GemvPlan g;
-    tman_status st = mpgemv_plan(M, K, N, count, bits, group, capacity9, &g);
-    if (st != TMAN_OK) return st;
-    const int v[16] = {g.mt, g.cluster, g.wpc, g.nkt, g.rpp, g.npass, g.ntiles, g.tpc, g.clusters, g.waves, g.stages,
-                       g.smem_bytes, g.tables_bytes, g.park_bytes, g.inbox_bytes, g.cost_clocks};
-    for (int i = 0; i < 16; ++i) out16[i] = v[i];
-    return TMAN_OK;
-}
-
 tman_status tman_debug_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer,
                                   size_t buffer_bytes, tman_stream_t stream)
 {

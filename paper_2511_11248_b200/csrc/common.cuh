@@ -107,32 +107,16 @@ __device__ __forceinline__ void lut16(float x0, float x1, float x2, float x3, fl
 // entry points implemented per file
 tman_status launch_pack(const uint8_t *codes, const void *scales, const uint8_t *zeros, int K, int N,
                         int bits, int group, void *packed, cudaStream_t s);
+// A packing on stream s is followed by one decode launch in plain stream order (no programmatic
+// dependent launch): note_packed_write records the stream, packed_write_pending asks and clears.
+void note_packed_write(cudaStream_t s);
+bool packed_write_pending(cudaStream_t s, bool clear);
 tman_status launch_unpack(const void *packed, int K, int N, int bits, int group, uint8_t *codes,
                           void *scales, uint8_t *zeros, uint32_t *status, cudaStream_t s);
 tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int group, uint8_t *idx,
                                  uint32_t *status, cudaStream_t s);
 tman_status launch_debug_luts(const void *x, int M, int K, float *lut, cudaStream_t s);
 size_t      mpgemv_workspace_bytes(int M, int K, int N);
-// How a decode call is cut (see plan_gemv in mpgemv.cu).
-struct GemvPlan {
-    int mt;            // activation rows a table entry carries (1, 2, 4, 8)
-    int cluster;       // CTAs per cluster = K-slices summed on chip
-    int wpc;           // plane words (32 activations) of a K-slice
-    int nkt;           // tile rows of a K-slice
-    int rpp;           // tile rows whose tables are resident at once
-    int npass;         // table builds per CTA
-    int ntiles;        // column tiles of the call
-    int tpc;           // column tiles per cluster
-    int clusters;      // clusters launched
-    int waves;         // rounds of resident clusters
-    int stages;        // ring depth (tiles)
-    int epc;           // output elements a CTA of a cluster finishes
-    int smem_bytes, tables_bytes, park_bytes, inbox_bytes, sums_bytes;
-    int sz_tma, nbt, zw, stage_bytes;   // scales and zero-points copied with the tile (1/0), blocks per tile row, zero-point row, stage size
-    int cost_clocks;   // the model's estimate for the busiest CTA
-};
-GemvPlan    plan_gemv(int M, int K, const int *Ns, int count, int bits, int group, const int *capacity);
-tman_status mpgemv_plan(int M, int K, const int *Ns, int count, int bits, int group, const int *capacity9, GemvPlan *out);
 tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s);
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s);

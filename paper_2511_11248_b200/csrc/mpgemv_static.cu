@@ -4,11 +4,11 @@
 // matmul: an inference runtime that sizes one arena at start-up and forbids cudaMalloc afterwards
 // (an allocation can synchronise the device and breaks a latency budget), a plug-in that runs inside
 // another framework's stream callback, code between "begin" and "end" of a region where the
-// allocator is locked.  tman_mpgemv needs scratch memory in global memory (the block that holds the
-// device-side status word; the K-slices themselves are summed on chip) that such a caller has nowhere
-// to put.  Here that scratch is a fixed array that is part of the library image: every GPU that
-// loads the library holds kStaticWsBytes of it from load until the process exits, and nothing is
-// allocated at call time.
+// allocator is locked.  tman_mpgemv needs scratch memory (a status word and the fp32
+// partial sums of the K-slices) that such a caller has nowhere to put.  Here that
+// scratch is a fixed array that is part of the library image: every GPU that loads the library
+// holds kStaticWsBytes of it from load until the process exits, and nothing is allocated at
+// call time.
 #include "common.cuh"
 
 #include <mutex>
@@ -16,7 +16,7 @@
 namespace tman {
 namespace {
 
-constexpr size_t kStaticWsBytes = 4096;               // 4 KiB per GPU
+constexpr size_t kStaticWsBytes = 4u << 20;          // 4 MiB per GPU
 constexpr int    kMaxDevices = 64;
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress: it is
@@ -69,7 +69,8 @@ extern "C" tman_status tman_mpgemv_static(const void *packed, size_t packed_byte
     st = static_ws(&ws);
     if (st != TMAN_OK) return st;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    // The array keeps whatever the last call left: the status word must start at zero.
+    // The array keeps whatever the last call left.  The status word must start at zero and the
+    // partial-sum area must say "no sum pending" everywhere this call will look.
     st = launch_workspace_init(ws, need, s);
     if (st != TMAN_OK) return st;
     st = launch_mpgemv(packed, x_f16, y_f16, M, K, N, bits, group, ws, kStaticWsBytes, s);

@@ -1,6 +1,9 @@
 // Offline repack into the bit-plane layout, its inverse, and the test-only extractors.
 // Pure integer work; every result has exactly one correct value.
 #include "common.cuh"
+#include <algorithm>
+#include <mutex>
+#include <vector>
 
 namespace tman {
 
@@ -79,6 +82,28 @@ __global__ void zero_padding_kernel(uint8_t *packed, int K, int N, int bits, int
     else { size_t t = tid - 512; if (c0 + t < c1) packed[c0 + t] = 0; }
 }
 
+// Streams on which a packed buffer has been written since the last decode launch.  The decode kernel
+// reads weights before it waits for its predecessor when launched with programmatic stream
+// serialization, so launch_mpgemv asks here and falls back to plain stream order once after a pack.
+static std::mutex g_pending_mutex;
+static std::vector<cudaStream_t> g_pending_streams;
+
+void note_packed_write(cudaStream_t s)
+{
+    std::lock_guard<std::mutex> lock(g_pending_mutex);
+    if (std::find(g_pending_streams.begin(), g_pending_streams.end(), s) == g_pending_streams.end())
+        g_pending_streams.push_back(s);
+}
+
+bool packed_write_pending(cudaStream_t s, bool clear)
+{
+    std::lock_guard<std::mutex> lock(g_pending_mutex);
+    auto it = std::find(g_pending_streams.begin(), g_pending_streams.end(), s);
+    if (it == g_pending_streams.end()) return false;
+    if (clear) g_pending_streams.erase(it);
+    return true;
+}
+
 tman_status launch_pack(const uint8_t *codes, const void *scales, const uint8_t *zeros, int K, int N,
                         int bits, int group, void *packed, cudaStream_t s)
 {
@@ -93,6 +118,7 @@ tman_status launch_pack(const uint8_t *codes, const void *scales, const uint8_t 
     pack_scales_kernel<<<(unsigned)((t2 + 255) / 256), 256, 0, s>>>(
         static_cast<const __half *>(scales), zeros, reinterpret_cast<__half *>(p + L.scales_off),
         reinterpret_cast<uint16_t *>(p + L.zeros_off), K, N, group);
+    note_packed_write(s);
     return launch_status();
 }
 

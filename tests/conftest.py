@@ -24,3 +24,15 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _guard_bytes_untouched(request):
+    """After every GPU test: no kernel wrote outside a buffer the helpers handed out."""
+    yield
+    if "gpu" in request.keywords:
+        import torch
+        if torch.cuda.is_available():
+            from paper_2511_11248_b200 import helpers
+            torch.cuda.synchronize()
+            helpers.check_guards(forget=True)

@@ -99,5 +99,5 @@ def test_workspace_sizes(lib):
     from paper_2511_11248_b200 import binding as B
     assert B.tman_workspace_bytes(B.OP_AUX, 1, 128, 8, 4, 64) == 256
     assert B.tman_workspace_bytes(B.OP_GEMM, 1024, 4096, 4096, 4, 128) >= 256
-    # decode sums its K-slices on chip: only the status block lives in the workspace
-    assert B.tman_workspace_bytes(B.OP_GEMV, 1, 4096, 4096, 4, 64) == 256
+    w = B.tman_workspace_bytes(B.OP_GEMV, 1, 4096, 4096, 4, 64)
+    assert w >= 256 + 4096 + 4 * 4096 * 4
