@@ -8,12 +8,18 @@ table build for both), down through a second call.  The packed weights rotate th
 whose total size exceeds L2, so every call streams from HBM.  Steps are replayed from a CUDA
 graph and timed with CUDA events on the launching stream.
 
-Also reported on the same JSON line: the prefill mpGEMM rate (M = 1024, K = 4096,
-N in {4096, 14336}, 4-bit, group 128) with its tensor roofline; the end-to-end rate through the
-C ABI with host buffers; the CPU oracle's rate on a bounded sample; clocks sampled during the
-timed region.
+The graph of 60 steps is replayed at least 20 times whatever --steps says; every replay is timed by its
+own pair of events, ms_per_step and value come from the median replay, and the line keeps the best
+replay and the replay count.
+
+Also reported on the same JSON line: under roofline.prefill the prefill mpGEMM rate (M = 1024,
+K = 4096, N in {4096, 14336}, 4-bit, group 128) with its tensor roofline; under roofline.ceilings the
+lookup-rate and instruction-issue ceilings of the decode kernel; under config one-line digests of
+configs 1, 3 and 5 measured in the same run; the end-to-end rate through the C ABI with host
+buffers; the CPU oracle's rate on a bounded sample; clocks sampled during the timed region.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py --leg {case,config1,config3,config5,microbench} [leg options]   # see bench_legs.py
 
 With N > 1 (launched under torchrun) every rank runs an independent replica of the same step
 (the path does not shard); value is the sum over ranks divided by the slowest rank's time.
@@ -40,6 +46,7 @@ MLP = [("gate", 4096, 14336), ("up", 4096, 14336), ("down", 14336, 4096)]
 BITS, GROUP = 2, 64
 NSETS = 6
 GRAPH_STEPS = 60
+MIN_REPLAYS = 20
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_FP16_TFLOPS = 2250.0
 FALLBACK_HBM_GBS = 6650.0
@@ -244,7 +251,7 @@ def run_ours(args):
     with torch.cuda.graph(graph):
         for i in range(GRAPH_STEPS):
             step(i)
-    n_replay = max(1, args.steps // GRAPH_STEPS)
+    n_replay = max(MIN_REPLAYS, -(-args.steps // GRAPH_STEPS))
     steps = n_replay * GRAPH_STEPS
     n_warm = max(1, -(-max(args.warmup, 3) // GRAPH_STEPS))
     for _ in range(n_warm):
@@ -257,16 +264,23 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_replay + 1)]
     barrier()
     with ClockSampler(physical_gpu_index(local_rank)) as clk:
         ev0.record()
-        for _ in range(n_replay):
+        marks[0].record()
+        for r in range(n_replay):
             graph.replay()
+            marks[r + 1].record()
         ev1.record()
         torch.cuda.synchronize()
     barrier()
-    ms = replicas.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
-    sec_step = ms / 1e3 / steps
+    # every replay's own duration: median for the headline, best and the whole region's mean beside it
+    replay_ms = np.array([marks[r].elapsed_time(marks[r + 1]) for r in range(n_replay)])
+    ms_median = replicas.max_over_ranks(float(np.median(replay_ms)), "cuda")
+    ms_best = replicas.max_over_ranks(float(np.min(replay_ms)), "cuda")
+    ms_total = replicas.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
+    sec_step = ms_median / 1e3 / GRAPH_STEPS
     value = replicas.whole_job_rate(wbytes_step, sec_step, world) / 1e9
     st = [B.tman_read_status(e[5]) for s in sets for e in s]
     assert all(v == 0 for v in st), f"device status {st}"
@@ -313,7 +327,7 @@ def run_ours(args):
     with torch.cuda.graph(e2e_graph):
         for i in range(GRAPH_STEPS):
             e2e_step(i, False)
-    e2e_replays = max(1, e2e_steps // GRAPH_STEPS)
+    e2e_replays = max(10, e2e_steps // GRAPH_STEPS)
     e2e_graph.replay()
     barrier()
     ev0.record()
@@ -384,7 +398,10 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
-        "warmup": n_warm * GRAPH_STEPS, "ms_per_step": sec_step * 1e3, "higher_is_better": True,
+        "warmup": n_warm * GRAPH_STEPS, "ms_per_step": sec_step * 1e3,
+        "ms_per_step_best": ms_best / GRAPH_STEPS, "ms_per_step_mean": ms_total / steps,
+        "replays": n_replay, "steps_per_replay": GRAPH_STEPS, "timing": "median over replays, each timed by its own events",
+        "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "replicas": world,
                    "l2": f"inputs larger than L2: {NSETS} rotating weight sets, {resident_mb:.0f} MB resident",
@@ -408,8 +425,13 @@ def run_ours(args):
                         "unit": "GB/s", "frac": ach / peaks["hbm"], "traffic": TRAFFIC_BYTES_PER_LAUNCH,
                         "peak_source": f"of {peaks['src']}", "algorithmic_bytes_per_launch": abytes_step / launches_per_step}
 
+    if rank == 0:
+        line["roofline"]["ceilings"] = decode_ceilings(torch, B, clk.summary(), abytes_step / launches_per_step, ach)
     if rank == 0 and not args.skip_gemm:
-        line["mpgemm"] = bench_gemm(torch, B, H, synth, peaks)
+        line["roofline"]["prefill"] = bench_gemm(torch, B, H, synth, peaks)
+    if rank == 0 and world == 1 and not args.skip_sweeps:
+        import bench_legs
+        line["config"].update(bench_legs.summaries(torch, B, H))
     if rank == 0 and world == 1 and not args.skip_cpu:
         line["cpu_baseline"] = cpu_baseline(host0, sets[0])
     if world > 1:
@@ -428,9 +450,41 @@ TRAFFIC_BYTES_PER_LAUNCH = 25171968.0 * (17.04 / 16.78)
 GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
 
 
+# Warp instructions the decode kernel executes for one gate/up-sized launch (16.78 MB of algorithmic
+# bytes), from the ncu capture summarised under profiles/ (smsp__inst_executed.sum).
+DECODE_WARP_INSTRUCTIONS_PER_BYTE = 3.56e6 / 16.78e6
+SCHEDULERS_PER_SM = 4
+
+
+def decode_ceilings(torch, B, clocks, bytes_per_launch, achieved_gbs):
+    """Two ceilings of the decode kernel other than HBM, in the units of roofline.achieved.
+    lookup: the rate at which one SM performs the kernel's lookup (8-bit index, 256-entry fp32 table in
+    shared memory, one add), measured now by the lookup microbenchmark; a lookup consumes one byte of a
+    bit plane, and planes are 8/9 (2-bit, group 64) of the bytes streamed.
+    issue: the kernel's warp instructions per byte (from its ncu capture) at one instruction per clock
+    per scheduler."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+    res = torch.zeros(8192, dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        res.zero_()
+        B.tman_debug_microbench(0, 512, res)
+    torch.cuda.synchronize()
+    clk = res[: sms * 8].view(torch.int64).cpu().numpy().astype(np.float64)
+    lookups_per_clk = float((1 << 20) / np.median(clk))
+    plane_share = (BITS / 8) / (BITS / 8 + (2 + BITS / 8) / GROUP)
+    lookup_gbs = lookups_per_clk * sms * mhz * 1e6 / plane_share / 1e9
+    issue_gbs = SCHEDULERS_PER_SM * sms * mhz * 1e6 / DECODE_WARP_INSTRUCTIONS_PER_BYTE / 1e9
+    return {"unit": "GB/s", "sm_mhz": mhz,
+            "lookup": {"lookups_per_clk_per_sm": round(lookups_per_clk, 2), "GBs": round(lookup_gbs, 1),
+                       "achieved_frac": round(achieved_gbs / lookup_gbs, 3)},
+            "issue": {"warp_instructions_per_byte": round(DECODE_WARP_INSTRUCTIONS_PER_BYTE, 4),
+                      "GBs": round(issue_gbs, 1), "achieved_frac": round(achieved_gbs / issue_gbs, 3)}}
+
+
 def bench_gemm(torch, B, H, synth, peaks):
     """Prefill mpGEMM, config 4: M=1024, K=4096, N in {4096, 14336}, 4-bit, group 128."""
-    out = {"unit": "TFLOP/s", "cases": []}
+    out = {"cases": []}
     tot_flops, tot_sec = 0.0, 0.0
     for spec in synth.config4_specs():
         c = synth.case_from_spec(spec)
@@ -459,11 +513,12 @@ def bench_gemm(torch, B, H, synth, peaks):
         tot_flops += flops
         tot_sec += sec
     tf = tot_flops / tot_sec / 1e12
-    out["value"] = tf
-    out["frac_of_nominal_fp16"] = tf / NOMINAL_FP16_TFLOPS
-    out["roofline"] = {"bound": "tensor", "kernel": "mpgemm_kernel<4,2,true> (4-bit, CTA pairs, two row blocks per CTA)", "achieved": tf, "peak": peaks["tf_burst"],
-                       "unit": "TFLOP/s", "frac": tf / peaks["tf_burst"], "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
-                       "peak_source": f"of {peaks['src']} (bf16 burst; fp16 has the same nominal rate)"}
+    out.update({"bound": "tensor", "kernel": "mpgemm_kernel<4,2,true> (4-bit, CTA pairs, two row blocks per CTA)",
+                "workload": "config4: prefill mpGEMM M=1024, K=4096, N in {4096, 14336}, 4-bit, group 128 "
+                            "(sum of flops / sum of time; 4 rotating copies of inputs and outputs, 40 calls each)",
+                "achieved": tf, "peak": peaks["tf_burst"], "unit": "TFLOP/s", "frac": tf / peaks["tf_burst"],
+                "frac_of_nominal_fp16": tf / NOMINAL_FP16_TFLOPS, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
+                "peak_source": f"of {peaks['src']} (bf16 burst; fp16 has the same nominal rate)"})
     return out
 
 
@@ -494,13 +549,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--skip-gemm", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
-    ap.add_argument("--leg", default="headline", choices=["headline", "microbench"],
+    ap.add_argument("--skip-sweeps", action="store_true", help="leave the config 1/3/5 digests out of the line")
+    ap.add_argument("--leg", default="headline", choices=["headline", "case", "config1", "config3", "config5", "microbench"],
                     help="headline: the bench line (default); the others print their own JSON lines")
-    args = ap.parse_args()
+    args, rest = ap.parse_known_args()
     if args.leg != "headline":
         import bench_legs
-        getattr(bench_legs, args.leg)(args)
+        getattr(bench_legs, args.leg)(args, rest)
         return
+    if rest:
+        ap.error(f"unknown arguments {rest}")
     if args.impl == "reference":
         run_reference(args)
     else:

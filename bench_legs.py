@@ -1,9 +1,21 @@
-"""Measurement legs that `bench.py --leg NAME` runs besides the headline step: the design
-microbenchmarks, a single shape (also the command line to profile), the decode batch sweep and the
-prefill shape sweep.  Everything goes through the C ABI; one JSON line per result on stdout.
+"""Measurement legs that `bench.py --leg NAME` runs besides the headline step:
+
+    python bench.py --leg case --op gemv --M 1 --K 4096 --N 14336 --bits 2 --group 64   # one shape (also the command to profile)
+    python bench.py --leg config1                  # decode, M=1, 4096x4096, 4-bit, group 64
+    python bench.py --leg config3 [--dense]        # one decoder layer's projections, bits {2,3,4} x M {1,2,4,8}
+    python bench.py --leg config5 [--dense] [--all-groups]   # prefill shapes, M in {128,512,2048,8192}
+    python bench.py --leg microbench               # lookup rates, load paths, cluster exchange
+
+Everything goes through the C ABI; one JSON line per result on stdout.  Weights and activations are
+seeded synthetic data drawn on the device (timing does not depend on the values; parity is the tests'
+business).  Weight sets rotate through copies whose total size exceeds L2, so every call streams from
+HBM.  With --dense a case also times the same product with fp16 weights through torch.matmul (the
+library GEMM/GEMV: a yardstick for what the low-bit weights buy or cost, not part of the path).
+The headline run calls summaries() for the one-line digests it carries.
 """
 from __future__ import annotations
 
+import argparse
 import json
 
 import numpy as np
@@ -11,6 +23,7 @@ import numpy as np
 L2_BYTES = 126e6
 LLAMA3_8B_LAYER = [("q", 4096, 4096), ("k", 4096, 1024), ("v", 4096, 1024), ("o", 4096, 4096),
                    ("gate", 4096, 14336), ("up", 4096, 14336), ("down", 14336, 4096)]
+QWEN25_7B_PROJ = [("gateup", 3584, 18944), ("down", 18944, 3584), ("qkv", 3584, 4608)]
 
 
 def weight_bytes(K, N, bits, group):
@@ -29,6 +42,270 @@ def event_us(torch, fn, reps):
     return float(np.median(ts)), float(np.min(ts))
 
 
+def device_problem(torch, B, H, M, K, N, bits, group, seed):
+    """Seeded synthetic weights (uniform codes and zero-points, scales in [0.005, 0.02]) packed by the
+    library, and activations ~ N(0, 1), all drawn on the device."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    codes = torch.randint(0, 1 << bits, (K, N), dtype=torch.uint8, device="cuda", generator=g)
+    zeros = torch.randint(0, 1 << bits, (K // group, N), dtype=torch.uint8, device="cuda", generator=g)
+    scales = (0.005 + 0.015 * torch.rand((K // group, N), device="cuda", generator=g)).to(torch.float16)
+    x = torch.randn((M, K), device="cuda", generator=g).to(torch.float16)
+    packed = torch.empty(B.tman_packed_bytes(K, N, bits, group), dtype=torch.uint8, device="cuda")
+    B.tman_pack_weights(codes, scales, zeros, K, N, bits, group, packed)
+    return packed, x
+
+
+def workspace(torch, B, op, M, K, N, bits, group):
+    ws = torch.empty(B.tman_workspace_bytes(op, M, K, N, bits, group), dtype=torch.uint8, device="cuda")
+    B.tman_workspace_init(ws)
+    return ws
+
+
+# ---- one shape -------------------------------------------------------------------------------------
+
+def case(args, rest=()):
+    import torch
+    from paper_2511_11248_b200 import binding as B, helpers as H
+    ap = argparse.ArgumentParser(prog="bench.py --leg case")
+    ap.add_argument("--op", choices=["gemv", "gemm"], default="gemv")
+    ap.add_argument("--M", type=int, default=1)
+    ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--N", type=int, default=4096)
+    ap.add_argument("--bits", type=int, default=4)
+    ap.add_argument("--group", type=int, default=64)
+    ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--copies", type=int, default=1, help="rotate over this many packed copies")
+    a = ap.parse_args(list(rest))
+    packed0, x = device_problem(torch, B, H, a.M, a.K, a.N, a.bits, a.group, seed=1)
+    packed = [packed0] + [packed0.clone() for _ in range(a.copies - 1)]
+    op = B.OP_GEMV if a.op == "gemv" else B.OP_GEMM
+    fn = B.tman_mpgemv if a.op == "gemv" else B.tman_mpgemm
+    ws = workspace(torch, B, op, a.M, a.K, a.N, a.bits, a.group)
+    y = torch.empty((a.M, a.N), dtype=torch.float16, device="cuda")
+    for i in range(3):
+        fn(packed[i % a.copies], x, y, a.M, a.K, a.N, a.bits, a.group, ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(a.iters):
+        fn(packed[i % a.copies], x, y, a.M, a.K, a.N, a.bits, a.group, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    assert B.tman_read_status(ws) == 0
+    us = e0.elapsed_time(e1) * 1e3 / a.iters
+    print(json.dumps({"leg": "case", "op": a.op, "M": a.M, "K": a.K, "N": a.N, "bits": a.bits, "group": a.group,
+                      "us_per_call": us, "iters": a.iters, "copies": a.copies}))
+
+
+# ---- decode: config 1 and the layer sweep (config 3) -------------------------------------------------
+
+def decode_calls_us(torch, B, H, M, bits, group, calls, reps):
+    """calls: list of lists of (K, N) that share activations (one grouped launch each).  Returns the
+    median and best time of one pass over all calls, replayed from a CUDA graph over rotating sets."""
+    pass_bytes = sum(weight_bytes(K, N, bits, group) for grp in calls for K, N in grp)
+    nsets = max(2, int(2.2 * L2_BYTES // pass_bytes) + 1)
+    sets = []
+    for s in range(nsets):
+        entry = []
+        for ci, grp in enumerate(calls):
+            K = grp[0][0]
+            packed, x = [], None
+            for gi, (_, N) in enumerate(grp):
+                p, xx = device_problem(torch, B, H, M, K, N, bits, group, seed=1000 * s + 10 * ci + gi)
+                packed.append(p)
+                x = xx if x is None else x
+            ys = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _, N in grp]
+            entry.append((K, [N for _, N in grp], packed, x, ys))
+        sets.append(entry)
+    wss = [workspace(torch, B, B.OP_GEMV, M, grp[0][0], sum(N for _, N in grp), bits, group) for grp in calls]
+
+    def one_pass(e):
+        for (K, Ns, packed, x, ys), ws in zip(e, wss):
+            if len(Ns) == 1:
+                B.tman_mpgemv(packed[0], x, ys[0], M, K, Ns[0], bits, group, ws)
+            else:
+                B.tman_mpgemv_grouped(packed, x, ys, M, K, Ns, bits, group, ws)
+
+    for e in sets:
+        one_pass(e)
+    torch.cuda.synchronize()
+    nrep = 4 * nsets
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(nrep):
+            one_pass(sets[i % nsets])
+    g.replay()
+    torch.cuda.synchronize()
+    med, best = event_us(torch, g.replay, reps)
+    assert all(B.tman_read_status(w) == 0 for w in wss)
+    return med / nrep, best / nrep, pass_bytes, nsets
+
+
+LAYER_CALLS = [[(4096, 4096), (4096, 1024), (4096, 1024)], [(4096, 4096)], [(4096, 14336), (4096, 14336)],
+               [(14336, 4096)]]
+
+
+def dense_layer_us(torch, M, reps):
+    """The layer's seven products with fp16 weights (torch.matmul), rotating weight sets > L2."""
+    layer_bytes = sum(K * N * 2 for _, K, N in LLAMA3_8B_LAYER)
+    nsets = max(2, int(2.2 * L2_BYTES // layer_bytes) + 1)
+    sets = [[(torch.randn((M, K), dtype=torch.float16, device="cuda"),
+              torch.randn((K, N), dtype=torch.float16, device="cuda") * 0.02) for _, K, N in LLAMA3_8B_LAYER]
+            for _ in range(nsets)]
+
+    def layer(e):
+        for x, w in e:
+            torch.matmul(x, w)
+
+    for e in sets:
+        layer(e)
+    torch.cuda.synchronize()
+    nrep = 4 * nsets
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(nrep):
+            layer(sets[i % nsets])
+    g.replay()
+    torch.cuda.synchronize()
+    return event_us(torch, g.replay, reps)[0] / nrep
+
+
+def config1_result(torch, B, H, reps=7):
+    med, best, nbytes, nsets = decode_calls_us(torch, B, H, 1, 4, 64, [[(4096, 4096)]], reps)
+    return {"leg": "config1", "M": 1, "K": 4096, "N": 4096, "bits": 4, "group": 64, "us": round(med, 2),
+            "us_best": round(best, 2), "weight_stream_GBs": round(nbytes / med / 1e3, 1), "weight_sets": nsets}
+
+
+def config1(args, rest=()):
+    import torch
+    from paper_2511_11248_b200 import binding as B, helpers as H
+    print(json.dumps(config1_result(torch, B, H)), flush=True)
+
+
+def config3_results(torch, B, H, reps=7, dense=False, bits_list=(2, 3, 4), Ms=(1, 2, 4, 8)):
+    out = []
+    dense_us = {M: dense_layer_us(torch, M, reps) for M in Ms} if dense else {}
+    torch.cuda.empty_cache()
+    for bits in bits_list:
+        for M in Ms:
+            med, best, nbytes, nsets = decode_calls_us(torch, B, H, M, bits, 128, LAYER_CALLS, reps)
+            r = {"leg": "config3", "M": M, "bits": bits, "group": 128, "layer_us": round(med, 2),
+                 "layer_us_best": round(best, 2), "weight_stream_GBs": round(nbytes / med / 1e3, 1),
+                 "weight_sets": nsets, "launches_per_layer": len(LAYER_CALLS)}
+            if dense:
+                r["dense_fp16_layer_us"] = round(dense_us[M], 2)
+                r["speedup_vs_dense_fp16"] = round(dense_us[M] / med, 2)
+            out.append(r)
+            torch.cuda.empty_cache()
+    return out
+
+
+def config3(args, rest=()):
+    import torch
+    from paper_2511_11248_b200 import binding as B, helpers as H
+    ap = argparse.ArgumentParser(prog="bench.py --leg config3")
+    ap.add_argument("--dense", action="store_true")
+    ap.add_argument("--reps", type=int, default=7)
+    a = ap.parse_args(list(rest))
+    for r in config3_results(torch, B, H, a.reps, a.dense):
+        print(json.dumps(r), flush=True)
+
+
+# ---- prefill shape sweep (config 5) --------------------------------------------------------------------
+
+def dense_case_us(torch, M, K, N, reps):
+    x = torch.randn((M, K), dtype=torch.float16, device="cuda")
+    ncopy = max(2, int(2.2 * L2_BYTES // (K * N * 2)) + 1)
+    ws = [torch.randn((K, N), dtype=torch.float16, device="cuda") * 0.02 for _ in range(ncopy)]
+    y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    for w in ws[:2]:
+        torch.matmul(x, w, out=y)
+    torch.cuda.synchronize()
+
+    def run():
+        for w in ws:
+            torch.matmul(x, w, out=y)
+
+    return event_us(torch, run, reps)[0] / ncopy
+
+
+def prefill_case(torch, B, H, M, K, N, bits, group, reps):
+    p0, x = device_problem(torch, B, H, M, K, N, bits, group, seed=5)
+    ncopy = max(2, int(2.2 * L2_BYTES // p0.numel()) + 1)
+    pk = [p0] + [p0.clone() for _ in range(ncopy - 1)]
+    ws = workspace(torch, B, B.OP_GEMM, M, K, N, bits, group)
+    ys = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in range(2)]
+    for i in range(3):
+        B.tman_mpgemm(pk[i % ncopy], x, ys[i % 2], M, K, N, bits, group, ws)
+    torch.cuda.synchronize()
+
+    def run():
+        for i in range(ncopy):
+            B.tman_mpgemm(pk[i], x, ys[i % 2], M, K, N, bits, group, ws)
+
+    us = event_us(torch, run, reps)[0] / ncopy
+    assert B.tman_read_status(ws) == 0
+    plan = B.tman_debug_gemm_plan(M, K, N, bits, group)
+    return {"leg": "config5", "M": M, "K": K, "N": N, "bits": bits, "group": group, "us": round(us, 1),
+            "TFLOPs": round(2.0 * M * K * N / us / 1e6, 1), "split_tiles": 1 - plan["whole_tiles"],
+            "column_tiles": plan["tiles_n"]}
+
+
+def config5_results(torch, B, H, reps=7, dense=False, bits_list=(2, 4), groups=(128,), Ms=(128, 512, 2048, 8192)):
+    out, dense_us = [], {}
+    for bits in bits_list:
+        for group in groups:
+            for M in Ms:
+                for _, K, N in QWEN25_7B_PROJ:
+                    r = prefill_case(torch, B, H, M, K, N, bits, group, reps)
+                    if dense:
+                        if (M, K, N) not in dense_us:
+                            dense_us[(M, K, N)] = dense_case_us(torch, M, K, N, reps)
+                        r["dense_fp16_us"] = round(dense_us[(M, K, N)], 1)
+                        r["time_vs_dense_fp16"] = round(r["us"] / dense_us[(M, K, N)], 2)
+                    out.append(r)
+                    torch.cuda.empty_cache()
+    return out
+
+
+def config5(args, rest=()):
+    import torch
+    from paper_2511_11248_b200 import binding as B, helpers as H
+    ap = argparse.ArgumentParser(prog="bench.py --leg config5")
+    ap.add_argument("--dense", action="store_true")
+    ap.add_argument("--all-groups", action="store_true", help="group 64 as well as 128")
+    ap.add_argument("--reps", type=int, default=7)
+    a = ap.parse_args(list(rest))
+    for r in config5_results(torch, B, H, a.reps, a.dense, groups=(64, 128) if a.all_groups else (128,)):
+        print(json.dumps(r), flush=True)
+
+
+# ---- digests for the headline line ------------------------------------------------------------------
+
+def summaries(torch, B, H):
+    """One-line digests of configs 1, 3 and 5, measured now: config 1 as [us, GB/s]; config 3 as layer
+    weight-stream GB/s per bits x M with the speed-up over fp16 weights through torch.matmul; config 5
+    as TFLOP/s per M (sum of flops / sum of time over the three shapes, group 128) per bit width with
+    the time relative to fp16 weights through torch.matmul."""
+    c1 = config1_result(torch, B, H, reps=5)
+    c3 = {}
+    for r in config3_results(torch, B, H, reps=5, dense=True):
+        c3.setdefault(f"b{r['bits']}", {})[f"M{r['M']}"] = [r["weight_stream_GBs"], r["speedup_vs_dense_fp16"]]
+    c5 = {}
+    rows = config5_results(torch, B, H, reps=3, dense=True)
+    for bits in (2, 4):
+        for M in (128, 512, 2048, 8192):
+            sel = [r for r in rows if r["bits"] == bits and r["M"] == M]
+            flops = sum(2.0 * r["M"] * r["K"] * r["N"] for r in sel)
+            us = sum(r["us"] for r in sel)
+            dus = sum(r["dense_fp16_us"] for r in sel)
+            c5.setdefault(f"b{bits}", {})[f"M{M}"] = [round(flops / us / 1e6, 1), round(us / dus, 2)]
+    return {"config1": {"us": c1["us"], "GBs": c1["weight_stream_GBs"]},
+            "config3": {"what": "[layer weight-stream GB/s, speed-up over fp16 torch.matmul], group 128", **c3},
+            "config5": {"what": "[TFLOP/s over the 3 shapes, time relative to fp16 torch.matmul], group 128", **c5}}
+
+
 # ---- design microbenchmarks ---------------------------------------------------------------------
 
 LOOKUP_KINDS = [
@@ -42,7 +319,7 @@ LOOKUP_KINDS = [
 ]
 
 
-def microbench(args):
+def microbench(args, rest=()):
     """Lookup rates per SM, load-path bandwidths, cluster exchange and L2 latency (one B200)."""
     import torch
     from paper_2511_11248_b200 import binding as B
