@@ -76,6 +76,7 @@ def case(args, rest=()):
     ap.add_argument("--group", type=int, default=64)
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--copies", type=int, default=1, help="rotate over this many packed copies")
+    ap.add_argument("--graph", action="store_true", help="time the calls replayed from one CUDA graph")
     a = ap.parse_args(list(rest))
     packed0, x = device_problem(torch, B, H, a.M, a.K, a.N, a.bits, a.group, seed=1)
     packed = [packed0] + [packed0.clone() for _ in range(a.copies - 1)]
@@ -83,19 +84,31 @@ def case(args, rest=()):
     fn = B.tman_mpgemv if a.op == "gemv" else B.tman_mpgemm
     ws = workspace(torch, B, op, a.M, a.K, a.N, a.bits, a.group)
     y = torch.empty((a.M, a.N), dtype=torch.float16, device="cuda")
+    def calls():
+        for i in range(a.iters):
+            fn(packed[i % a.copies], x, y, a.M, a.K, a.N, a.bits, a.group, ws)
+
     for i in range(3):
         fn(packed[i % a.copies], x, y, a.M, a.K, a.N, a.bits, a.group, ws)
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(a.iters):
-        fn(packed[i % a.copies], x, y, a.M, a.K, a.N, a.bits, a.group, ws)
-    e1.record()
-    torch.cuda.synchronize()
+    if a.graph:
+        # back-to-back calls without host launch cost: what a call takes inside a decoding step
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            calls()
+        g.replay()
+        torch.cuda.synchronize()
+        us = event_us(torch, g.replay, 7)[0] / a.iters
+    else:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        calls()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / a.iters
     assert B.tman_read_status(ws) == 0
-    us = e0.elapsed_time(e1) * 1e3 / a.iters
     print(json.dumps({"leg": "case", "op": a.op, "M": a.M, "K": a.K, "N": a.N, "bits": a.bits, "group": a.group,
-                      "us_per_call": us, "iters": a.iters, "copies": a.copies}))
+                      "us_per_call": round(us, 2), "iters": a.iters, "copies": a.copies, "graph": bool(a.graph)}))
 
 
 # ---- decode: config 1 and the layer sweep (config 3) -------------------------------------------------
