@@ -149,6 +149,20 @@ __device__ __forceinline__ void lookup_rows(uint32_t off, float (&out)[MT])
     }
 }
 
+// The same lookup returning the raw 32-bit slots (two fp16 rows each).
+template <int MT, uint32_t IMM>
+__device__ __forceinline__ void lookup_slots(uint32_t off, uint32_t (&out)[MT])
+{
+    if constexpr (MT == 1) {
+        asm volatile("ld.shared.b32 %0, [%1 + %2];" : "=r"(out[0]) : "r"(off), "n"(IMM));
+    } else if constexpr (MT == 2) {
+        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2 + %3];" : "=r"(out[0]), "=r"(out[1]) : "r"(off), "n"(IMM));
+    } else {
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4 + %5];"
+                     : "=r"(out[0]), "=r"(out[1]), "=r"(out[2]), "=r"(out[3]) : "r"(off), "n"(IMM));
+    }
+}
+
 // One unit's worth of a lane's inputs: its plane word of S strips, and the strips' scales and
 // zero-points of the lane's quantization block.
 template <int BITS, int S>
@@ -168,16 +182,23 @@ struct UnitRegs {
 // visits the index bytes of a word in the order 1,0,3,2, so that the 32 lanes still address 32
 // different banks.
 // GROUPED = 0: one matrix, the matrix index is a compile-time zero.
+// HR (more than one activation row): a 32-bit table slot holds two rows as fp16 instead of one as fp32,
+// so an entry of MT slots serves 2 * MT rows for the same shared-memory traffic.  Each row of the
+// K-slice is first scaled by a power of two that brings its largest magnitude into [1, 2) (undone in
+// fp32 at the end), so that entries use fp16's range whatever the activations' size; the bits * 4
+// lookups of one plane word are accumulated in fp16 (low plane first), everything after that in fp32.
 // ROLL: one set of unit registers; every strip's registers are refilled with the next unit's strip as
 // soon as its lookups are done (larger units, fewer per-unit fixed costs, same bytes in flight).
-template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL>
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL, int HR>
 __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     static_assert(!HALF || MT == 1, "half slices are for single-row tables");
+    static_assert(!HR || !HALF, "fp16 row pairs use whole-warp or sub-warp slices");
+    constexpr int R = HR ? 2 * MT : MT;    // activation rows of this launch
     constexpr int W = HALF ? 16 : 32 / MT; // plane words (lanes) per K-slice
     constexpr int SUBS = 32 / W;           // sub-warps, each on its own strips
-    constexpr int V = 4 * S * MT;         // values a lane produces per warp-unit
+    constexpr int V = 4 * S * R;          // values a lane produces per warp-unit
     constexpr int V1 = PRE ? V / 2 : V;   // values it still holds when scales are applied
     constexpr int NKEEP = (V >= W) ? V / W : 1;
 
@@ -296,6 +317,69 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
             for (int e = 0; e < 16; ++e) *reinterpret_cast<float *>(dst + (q * 16 + e) * 256) = lo[e] + base;
         }
+    } else if constexpr (HR) {
+        // The activations of this thread's table slot: one plane word = 32 activations of rows 2*mb and 2*mb+1.
+        const int vb = lane / MT, mb = lane % MT;
+        uint4 xraw[2][4];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const bool live = (vb < nwords) && (2 * mb + r < p.M);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) xraw[r][c] = make_uint4(0u, 0u, 0u, 0u);
+            if (live) {
+                const uint4 *px = reinterpret_cast<const uint4 *>(p.x + (size_t)(2 * mb + r) * p.K + (size_t)(word0 + vb) * 32);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) xraw[r][c] = __ldg(px + c);
+            }
+        }
+        if constexpr (!ROLL) load_unit(regs[1], wu0 + wstride);
+
+        // largest magnitude of each row over the K-slice -> power-of-two scale (every warp computes the same)
+        float inv[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            __half2 mx = __floats2half2_rn(0.f, 0.f);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const __half2 *h = reinterpret_cast<const __half2 *>(&xraw[r][c]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) mx = __hmax2(mx, __habs2(h[q]));
+            }
+            float amax = fmaxf(__low2float(mx), __high2float(mx));
+#pragma unroll
+            for (int mask = MT; mask < 32; mask <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, mask));
+            const uint32_t e = (__float_as_uint(amax) >> 23) & 0xFFu;      // amax = 1.f * 2^(e - 127)
+            inv[r] = __uint_as_float((254u - e) << 23);
+            if (warp == 0 && vb == 0)
+                reinterpret_cast<float *>(smem + kGemvTableBytes)[2 * mb + r] = __uint_as_float(e << 23);
+        }
+        {
+            const int ph = warp;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float lo[2][16], hi[2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    float xv[8];
+#pragma unroll
+                    for (int qq = 0; qq < 4; ++qq) {
+                        const float2 f = __half22float2(reinterpret_cast<const __half2 *>(&xraw[r][qq])[c]);
+                        xv[qq] = f.x * inv[r];
+                        xv[qq + 4] = f.y * inv[r];
+                    }
+                    lut16(xv[0], xv[1], xv[2], xv[3], lo[r]);
+                    hi[r] = 0.f;
+                    if (ph & 1) hi[r] += xv[4];
+                    if (ph & 2) hi[r] += xv[5];
+                    if (ph & 4) hi[r] += xv[6];
+                    if (ph & 8) hi[r] += xv[7];
+                }
+                uint8_t *dst = smem + table_imm(c) + (uint32_t)(ph * 16) * 256u + (uint32_t)lane * 4u;
+#pragma unroll
+                for (int pl = 0; pl < 16; ++pl)
+                    *reinterpret_cast<__half2 *>(dst + pl * 256) = __floats2half2_rn(lo[0][pl] + hi[0], lo[1][pl] + hi[1]);
+            }
+        }
     } else {
         // The activations of this thread's table slot (one plane word = 32 activations of one row).
         const int vb = lane / MT, mb = lane % MT;
@@ -360,21 +444,31 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     uint32_t sel_h[4];
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) sel_h[jj] = 0x7604u | ((uint32_t)(jj ^ sub) << 4);
-    float ssum[MT];
+    float ssum[R];
     {
 #pragma unroll
-        for (int m = 0; m < MT; ++m) ssum[m] = 0.f;
+        for (int m = 0; m < R; ++m) ssum[m] = 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            float t[MT];
-            if constexpr (HALF) load_rows<MT>(smem + 255u * 256u + (uint32_t)(v + 16 * c) * 4u, t);
-            else load_rows<MT>(smem + table_imm(c) + 255u * 256u + sub_off, t);
+            if constexpr (HR) {
 #pragma unroll
-            for (int m = 0; m < MT; ++m) ssum[m] += t[m];
+                for (int m = 0; m < MT; ++m) {
+                    const float2 f = __half22float2(
+                        *reinterpret_cast<const __half2 *>(smem + table_imm(c) + 255u * 256u + sub_off + 4u * m));
+                    ssum[2 * m] += f.x;
+                    ssum[2 * m + 1] += f.y;
+                }
+            } else {
+                float t[MT];
+                if constexpr (HALF) load_rows<MT>(smem + 255u * 256u + (uint32_t)(v + 16 * c) * 4u, t);
+                else load_rows<MT>(smem + table_imm(c) + 255u * 256u + sub_off, t);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) ssum[m] += t[m];
+            }
         }
         if constexpr (PRE) {
 #pragma unroll
-            for (int m = 0; m < MT; ++m) ssum[m] += __shfl_xor_sync(0xffffffffu, ssum[m], 1);
+            for (int m = 0; m < R; ++m) ssum[m] += __shfl_xor_sync(0xffffffffu, ssum[m], 1);
         }
     }
 
@@ -394,15 +488,23 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
                 float a[MT];
+                __half2 a2[MT];
 #pragma unroll
-                for (int m = 0; m < MT; ++m) a[m] = 0.f;
+                for (int m = 0; m < MT; ++m) { a[m] = 0.f; a2[m] = __floats2half2_rn(0.f, 0.f); }
 #pragma unroll
                 for (int i = 0; i < BITS; ++i) {
                     const uint32_t w = (c4 == 0) ? r.w[s][i].x : (c4 == 1) ? r.w[s][i].y
                                      : (c4 == 2) ? r.w[s][i].z : r.w[s][i].w;
+                    const __half2 pw = __floats2half2_rn((float)(1 << i), (float)(1 << i));
                     // byte 1 <- index byte c of the word, byte 0 <- the lane's slot offset
 #define TMAN_LOOKUP(c)                                                                          \
-    {                                                                                           \
+    if constexpr (HR) {                                                                         \
+        uint32_t t[MT];                                                                         \
+        const uint32_t off = __byte_perm(w, sub_off, 0x7604u | ((uint32_t)(c) << 4));           \
+        lookup_slots<MT, kGemvSmemBase + table_imm(c)>(off, t);                                 \
+        _Pragma("unroll") for (int m = 0; m < MT; ++m)                                          \
+            a2[m] = __hfma2(*reinterpret_cast<const __half2 *>(&t[m]), pw, a2[m]);              \
+    } else {                                                                                    \
         float t[MT];                                                                            \
         if constexpr (HALF) {                                                                   \
             const uint32_t off = __byte_perm(w, ((c) & 1) ? off_odd : off_even, sel_h[c]);      \
@@ -416,8 +518,17 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                     TMAN_LOOKUP(0) TMAN_LOOKUP(1) TMAN_LOOKUP(2) TMAN_LOOKUP(3)
 #undef TMAN_LOOKUP
                 }
+                if constexpr (HR) {
 #pragma unroll
-                for (int m = 0; m < MT; ++m) vals[(s * 4 + c4) * MT + m] = a[m];
+                    for (int m = 0; m < MT; ++m) {
+                        const float2 f = __half22float2(a2[m]);
+                        vals[(s * 4 + c4) * R + 2 * m] = f.x;
+                        vals[(s * 4 + c4) * R + 2 * m + 1] = f.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) vals[(s * 4 + c4) * MT + m] = a[m];
+                }
             }
             if constexpr (ROLL) load_strip(r, s, nxt);
         }
@@ -440,8 +551,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 for (int c4 = 0; c4 < 4; ++c4) {
                     const float zf = (float)((zq >> (4 * c4)) & 0xFu);
 #pragma unroll
-                    for (int m = 0; m < MT; ++m) {
-                        float &val = vals[(s * 4 + c4) * MT + m];
+                    for (int m = 0; m < R; ++m) {
+                        float &val = vals[(s * 4 + c4) * R + m];
                         val = sc[c4] * fmaf(-zf, ssum[m], val);
                     }
                 }
@@ -456,8 +567,8 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             for (int c2 = 0; c2 < 2; ++c2) {
                 const float zf = (float)((zq >> (4 * c2)) & 0xFu);
 #pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    float &val = vals[c2 * MT + m];
+                for (int m = 0; m < R; ++m) {
+                    float &val = vals[c2 * R + m];
                     val = sc[c2] * fmaf(-zf, ssum[m], val);
                 }
             }
@@ -470,10 +581,12 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             const int lim = GROUPED ? p.col0[g] + p.Ng[g] : p.N;   // end of this matrix's columns
 #pragma unroll
             for (int e = 0; e < NKEEP; ++e) {
-                const int idx = base + e, m = idx % MT, n = col_u + idx / MT;
+                const int idx = base + e, m = idx % R, n = col_u + idx / R;
                 if (n < lim && m < p.M) {
-                    if (p.nkappa == 1) p.y[g][(size_t)m * p.Ng[g] + (n - (GROUPED ? p.col0[g] : 0))] = __float2half_rn(vals[e]);
-                    else p.partials[((size_t)kappa * MT + m) * p.N + n] = vals[e];
+                    float out = vals[e];
+                    if constexpr (HR) out *= reinterpret_cast<const float *>(smem + kGemvTableBytes)[m];   // undo the row's scale
+                    if (p.nkappa == 1) p.y[g][(size_t)m * p.Ng[g] + (n - (GROUPED ? p.col0[g] : 0))] = __float2half_rn(out);
+                    else p.partials[((size_t)kappa * R + m) * p.N + n] = out;
                 }
             }
         }
@@ -499,7 +612,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         const int col_lo = g_lo * 4;
         const int ngrp = g_hi - g_lo;
         const int items = ngrp * p.M;                       // one item = four columns of one row
-        const size_t stride4 = (size_t)MT * p.N / 4;
+        const size_t stride4 = (size_t)R * p.N / 4;
         // SP adjacent lanes share an item and split the slices among them (slice kp goes to lane
         // kp % SP); their sums are added in a fixed order, so the result does not depend on timing
         int SP = 1;
@@ -557,12 +670,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     }
 }
 
-template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL>
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL, int HR>
 static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
 {
     constexpr int W = HALF ? 16 : 32 / MT;
     constexpr int SUBS = 32 / W;
-    constexpr int kSmem = HALF ? kGemvTableBytes / 2 : kGemvTableBytes;
+    // fp16 row pairs: the rows' scales follow the tables
+    constexpr int kSmem = HALF ? kGemvTableBytes / 2 : kGemvTableBytes + (HR ? 64 : 0);
     const int words_total = p.K / 32;
     p.nkappa = (words_total + W - 1) / W;
     p.P = sms / p.nkappa;
@@ -581,7 +695,7 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
         cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev) != cudaSuccess)
         return TMAN_ERR_CUDA;
     if ((uint32_t)reserved != kGemvSmemBase) return TMAN_ERR_UNSUPPORTED;
-    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED, ROLL>;
+    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED, ROLL, HR>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
         return TMAN_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -600,14 +714,27 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     return TMAN_OK;
 }
 
-template <int BITS, int MT, int PRE>
+template <int BITS, int MT, int PRE, int HR>
 static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
 {
-    // one row: large units on one rolling set of registers; more rows: small double-buffered units
-    constexpr int ROLL = (MT == 1) ? 1 : 0;
-    constexpr int S = (MT == 1) ? ((BITS == 2) ? 4 : 2) : 1;
-    if (p.count > 1) return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 1, ROLL>(p, sms, s);
-    return launch_one<BITS, MT, S, PRE, (MT == 1) ? 1 : 0, 0, ROLL>(p, sms, s);
+    // one row: fp32 tables over half-warp slices, large units on one rolling set of registers;
+    // more rows: fp16 row pairs, small double-buffered units
+    constexpr int ROLL = HR ? 0 : 1;
+    constexpr int S = HR ? 1 : ((BITS == 2) ? 4 : 2);
+    constexpr int HALF = HR ? 0 : 1;
+    if (p.count > 1) return launch_one<BITS, MT, S, PRE, HALF, 1, ROLL, HR>(p, sms, s);
+    return launch_one<BITS, MT, S, PRE, HALF, 0, ROLL, HR>(p, sms, s);
+}
+
+// Rows a launch carries and plane words per K-slice, by the number of rows in the call: 1 row -> fp32
+// tables, 16 words; 2 rows -> one fp16 pair per entry, 32 words; 3-4 rows -> two pairs, 16 words;
+// 5-8 rows -> four pairs, 8 words.
+static void gemv_variant(int M, int *rows, int *words)
+{
+    if (M <= 1) { *rows = 1; *words = 16; }
+    else if (M == 2) { *rows = 2; *words = 32; }
+    else if (M <= 4) { *rows = 4; *words = 16; }
+    else { *rows = 8; *words = 8; }
 }
 
 template <int BITS>
@@ -615,9 +742,10 @@ static tman_status launch_rows(GemvParams p, int rows, int sms, cudaStream_t s)
 {
     p.M = rows;
     const bool pre = p.group >= 64;
-    if (rows == 1) return pre ? launch_mt<BITS, 1, 1>(p, sms, s) : launch_mt<BITS, 1, 0>(p, sms, s);
-    if (rows == 2) return pre ? launch_mt<BITS, 2, 1>(p, sms, s) : launch_mt<BITS, 2, 0>(p, sms, s);
-    return pre ? launch_mt<BITS, 4, 1>(p, sms, s) : launch_mt<BITS, 4, 0>(p, sms, s);
+    if (rows == 1) return pre ? launch_mt<BITS, 1, 1, 0>(p, sms, s) : launch_mt<BITS, 1, 0, 0>(p, sms, s);
+    if (rows == 2) return pre ? launch_mt<BITS, 1, 1, 1>(p, sms, s) : launch_mt<BITS, 1, 0, 1>(p, sms, s);
+    if (rows <= 4) return pre ? launch_mt<BITS, 2, 1, 1>(p, sms, s) : launch_mt<BITS, 2, 0, 1>(p, sms, s);
+    return pre ? launch_mt<BITS, 4, 1, 1>(p, sms, s) : launch_mt<BITS, 4, 0, 1>(p, sms, s);
 }
 
 __global__ void ws_fill_kernel(uint32_t *ws, size_t words)
@@ -636,10 +764,11 @@ tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s)
 
 size_t mpgemv_workspace_bytes(int M, int K, int N)
 {
-    (void)M;
-    // worst case: rows are processed four at a time with K-slices of 8 plane words
-    const size_t nkappa = (size_t)(K / 32 + 7) / 8;
-    return kWsStatusBytes + nkappa * 4 * (size_t)N * sizeof(float);
+    // one fp32 partial sum per K-slice, row of the launch and column
+    int rows = 1, words = 16;
+    gemv_variant(M, &rows, &words);
+    const size_t nkappa = (size_t)(K / 32 + words - 1) / (size_t)words;
+    return kWsStatusBytes + nkappa * (size_t)rows * (size_t)N * sizeof(float);
 }
 
 tman_status launch_mpgemv_grouped(int count, const void *const *packed, const void *x, void *const *y, int M, int K,
@@ -671,9 +800,9 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
     p.M = 0; p.nkappa = 0; p.P = 0; p.units = 0;
     p.group_shift = (group == 32) ? 5 : (group == 64) ? 6 : 7;
     p.nblk = K / group;
-    // rows go through in batches of at most four (a table entry carries up to four rows)
-    for (int m0 = 0; m0 < M; m0 += 4) {
-        const int rows = (M - m0 < 4) ? (M - m0) : 4;
+    // a table entry carries up to eight rows (four fp16 pairs): one pass over the weights for M <= 8
+    for (int m0 = 0; m0 < M; m0 += 8) {
+        const int rows = (M - m0 < 8) ? (M - m0) : 8;
         p.x = static_cast<const __half *>(x) + (size_t)m0 * K;
         for (int g = 0; g < kGemvMaxGroup; ++g)
             p.y[g] = static_cast<__half *>(y[g < count ? g : 0]) + (size_t)m0 * p.Ng[g];

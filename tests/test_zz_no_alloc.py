@@ -99,12 +99,12 @@ def test_status_word_reaches_the_caller_and_a_good_call_follows_a_refused_one():
 
 
 def test_shape_beyond_the_fixed_array_is_refused():
-    # scratch for K = 18944, N = 18944 is far above 4 MiB: refused on the host, nothing enqueued
-    K, N, bits, G = 18944, 18944, 2, 128
-    assert B.tman_workspace_bytes(B.OP_GEMV, 1, K, N, bits, G) > (4 << 20)
+    # scratch for four rows, K = 18944, N = 18944 is far above 4 MiB: refused on the host, nothing enqueued
+    M, K, N, bits, G = 4, 18944, 18944, 2, 128
+    assert B.tman_workspace_bytes(B.OP_GEMV, M, K, N, bits, G) > (4 << 20)
     packed = torch.empty(B.tman_packed_bytes(K, N, bits, G), dtype=torch.uint8, device="cuda")
-    x = torch.zeros((1, K), dtype=torch.float16, device="cuda")
-    y = torch.zeros((1, N), dtype=torch.float16, device="cuda")
+    x = torch.zeros((M, K), dtype=torch.float16, device="cuda")
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
     with pytest.raises(B.TmanError) as e:
-        B.tman_mpgemv_static(packed, x, y, 1, K, N, bits, G)
+        B.tman_mpgemv_static(packed, x, y, M, K, N, bits, G)
     assert e.value.status == 4   # TMAN_ERR_BUFFER_TOO_SMALL
