@@ -196,6 +196,14 @@ tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_st
  * know which path a shape takes. */
 tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *out8 /*host*/);
 
+/* The same decision for a device described by the caller: `sms` multiprocessors, of which `resident`
+ * workers (CTAs, or CTA pairs when pairs are used) of the kernel can run at the same time.  The
+ * workers of a call wait for one another's partial tiles, so a call never launches more than
+ * `resident` of them; tman_mpgemm takes that number from the occupancy query of the kernel it is about
+ * to launch.  Pure host arithmetic: needs no GPU. */
+tman_status tman_debug_gemm_plan_for(int M, int K, int N, int bits, int group, int sms, int resident,
+                                     int *out8 /*host*/);
+
 /* Microbenchmarks behind the decode kernel's design, the counterpart on this GPU of the paper's
  * instruction study (Sec. 5 "Implementation", Table 1: lookups per instruction x log2(table entries) =
  * "equivalent multiply-adds" of the 16- and 32-entry lookup instructions) and of its load-path study

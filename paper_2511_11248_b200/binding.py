@@ -23,7 +23,7 @@ EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
     "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
-    "tman_debug_microbench", "tman_debug_cluster_capacity",
+    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for",
 ]
 
 _lib = None
@@ -170,6 +170,12 @@ def tman_debug_indices(packed, K, N, bits, group, idx, workspace, stream=None) -
 def tman_debug_gemm_plan(M, K, N, bits, group) -> dict:
     out = (C.c_int * 8)()
     _check(lib().tman_debug_gemm_plan(M, K, N, bits, group, out), "tman_debug_gemm_plan")
+    return dict(zip(("pair", "row_blocks", "tiles_m", "tiles_n", "whole_tiles", "workers", "span_tiles", "pieces"), list(out)))
+
+
+def tman_debug_gemm_plan_for(M, K, N, bits, group, sms, resident) -> dict:
+    out = (C.c_int * 8)()
+    _check(lib().tman_debug_gemm_plan_for(M, K, N, bits, group, sms, resident, out), "tman_debug_gemm_plan_for")
     return dict(zip(("pair", "row_blocks", "tiles_m", "tiles_n", "whole_tiles", "workers", "span_tiles", "pieces"), list(out)))
 
 

@@ -4,6 +4,13 @@
 
 using namespace tman;
 
+// Alignment rules of the header, in one place: packed buffers and workspaces start on a 256-byte
+// boundary, activation and output matrices on a 16-byte boundary.  Checked on the host before anything
+// touches the GPU; a violation is TMAN_ERR_SHAPE.
+static bool aligned_to(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+static bool buffers_aligned(const void *packed, const void *workspace) { return aligned_to(packed, 256) && aligned_to(workspace, 256); }
+static bool matrices_aligned(const void *x, const void *y) { return aligned_to(x, 16) && aligned_to(y, 16); }
+
 extern "C" {
 
 const char *tman_status_string(int status)
@@ -56,13 +63,14 @@ tman_status tman_workspace_init(void *workspace, size_t ws_bytes, tman_stream_t 
 {
     if (!workspace) return TMAN_ERR_NULL;
     if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
-    if (reinterpret_cast<uintptr_t>(workspace) & 255) return TMAN_ERR_SHAPE;
+    if (!aligned_to(workspace, 256)) return TMAN_ERR_SHAPE;
     return launch_workspace_init(workspace, ws_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
 tman_status tman_read_status(const void *workspace, int *out_status, tman_stream_t stream)
 {
     if (!workspace || !out_status) return TMAN_ERR_NULL;
+    if (!aligned_to(workspace, 256)) return TMAN_ERR_SHAPE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     uint32_t v = 0;
     if (cudaMemcpyAsync(&v, workspace, sizeof(v), cudaMemcpyDeviceToHost, s) != cudaSuccess) return TMAN_ERR_CUDA;
@@ -79,7 +87,7 @@ tman_status tman_pack_weights(const uint8_t *codes, const void *scales_f16, cons
     tman_status st = check_format(K, N, bits, group);
     if (st != TMAN_OK) return st;
     if (packed_bytes < make_layout(K, N, bits, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
-    if (reinterpret_cast<uintptr_t>(packed) & 255) return TMAN_ERR_SHAPE;
+    if (!aligned_to(packed, 256)) return TMAN_ERR_SHAPE;
     return launch_pack(codes, scales_f16, zeros, K, N, bits, group, packed, reinterpret_cast<cudaStream_t>(stream));
 }
 
@@ -93,6 +101,7 @@ tman_status tman_unpack_weights(const void *packed, size_t packed_bytes,
     if (st != TMAN_OK) return st;
     if (packed_bytes < make_layout(K, N, bits, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
     if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (!buffers_aligned(packed, workspace)) return TMAN_ERR_SHAPE;
     return launch_unpack(packed, K, N, bits, group, codes, scales_f16, zeros,
                          static_cast<uint32_t *>(workspace), reinterpret_cast<cudaStream_t>(stream));
 }
@@ -106,7 +115,7 @@ static tman_status check_matmul(const void *packed, size_t packed_bytes, const v
     if (packed_bytes < make_layout(K, N, bits, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
     if (bits < 2) return TMAN_ERR_UNSUPPORTED;
     if (M < 1) return TMAN_ERR_SHAPE;
-    if (reinterpret_cast<uintptr_t>(packed) & 255) return TMAN_ERR_SHAPE;
+    if (!buffers_aligned(packed, ws) || !matrices_aligned(x, y)) return TMAN_ERR_SHAPE;
     return TMAN_OK;
 }
 
@@ -117,9 +126,6 @@ tman_status tman_mpgemv(const void *packed, size_t packed_bytes, const void *x_f
     tman_status st = check_matmul(packed, packed_bytes, x_f16, y_f16, M, K, N, bits, group, workspace);
     if (st != TMAN_OK) return st;
     if (M > 8) return TMAN_ERR_SHAPE;
-    if ((reinterpret_cast<uintptr_t>(x_f16) & 15) || (reinterpret_cast<uintptr_t>(y_f16) & 15) ||
-        (reinterpret_cast<uintptr_t>(workspace) & 255))
-        return TMAN_ERR_SHAPE;
     if (ws_bytes < mpgemv_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
     return launch_mpgemv(packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
                          reinterpret_cast<cudaStream_t>(stream));
@@ -135,11 +141,9 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed, const size
     for (int g = 0; g < count; ++g) {
         tman_status st = check_matmul(packed[g], packed_bytes[g], x_f16, y_f16[g], M, K, N[g], bits, group, workspace);
         if (st != TMAN_OK) return st;
-        if (reinterpret_cast<uintptr_t>(y_f16[g]) & 15) return TMAN_ERR_SHAPE;
         ntot += N[g];
     }
     if (M > 8 || ntot > (1 << 30)) return TMAN_ERR_SHAPE;
-    if ((reinterpret_cast<uintptr_t>(x_f16) & 15) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return TMAN_ERR_SHAPE;
     if (ws_bytes < mpgemv_workspace_bytes(M, K, (int)ntot)) return TMAN_ERR_BUFFER_TOO_SMALL;
     return launch_mpgemv_grouped(count, packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
                                  reinterpret_cast<cudaStream_t>(stream));
@@ -163,6 +167,7 @@ tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int g
     tman_status st = check_format(K, N, bits, group);
     if (st != TMAN_OK) return st;
     if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (!buffers_aligned(packed, workspace)) return TMAN_ERR_SHAPE;
     return launch_debug_indices(packed, K, N, bits, group, idx, static_cast<uint32_t *>(workspace),
                                 reinterpret_cast<cudaStream_t>(stream));
 }
@@ -180,15 +185,25 @@ tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *
     tman_status st = check_format(K, N, bits, group);
     if (st != TMAN_OK) return st;
     if (M < 1) return TMAN_ERR_SHAPE;
-    return mpgemm_plan(M, K, N, out8);
+    if (bits < 2) return TMAN_ERR_UNSUPPORTED;
+    return mpgemm_plan(M, K, N, bits, out8);
+}
+
+tman_status tman_debug_gemm_plan_for(int M, int K, int N, int bits, int group, int sms, int resident, int *out8)
+{
+    if (!out8) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    if (M < 1 || sms < 1 || resident < 1) return TMAN_ERR_SHAPE;
+    if (bits < 2) return TMAN_ERR_UNSUPPORTED;
+    return mpgemm_plan_for(M, K, N, bits, sms, resident, out8);
 }
 
 tman_status tman_debug_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer,
                                   size_t buffer_bytes, tman_stream_t stream)
 {
     if (!results) return TMAN_ERR_NULL;
-    if (results_bytes < 4096 || (reinterpret_cast<uintptr_t>(results) & 255) || (reinterpret_cast<uintptr_t>(buffer) & 255))
-        return TMAN_ERR_SHAPE;
+    if (results_bytes < 4096 || !buffers_aligned(results, buffer)) return TMAN_ERR_SHAPE;
     return launch_microbench(kind, arg, results, results_bytes, buffer, buffer_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 

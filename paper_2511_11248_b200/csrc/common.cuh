@@ -123,7 +123,8 @@ tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int
 tman_status launch_mpgemv_grouped(int count, const void *const *packed, const void *x, void *const *y, int M, int K,
                                   const int *Ns, int bits, int group, void *ws, size_t ws_bytes, cudaStream_t s);
 size_t      mpgemm_workspace_bytes(int M, int K, int N);
-tman_status mpgemm_plan(int M, int K, int N, int *out8);
+tman_status mpgemm_plan(int M, int K, int N, int bits, int *out8);
+tman_status mpgemm_plan_for(int M, int K, int N, int bits, int sms, int resident, int *out8);
 tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s);
 tman_status launch_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer, size_t buffer_bytes,

@@ -31,6 +31,8 @@
 // work, and still reaches the common tear-down that frees tensor memory.
 #include "common.cuh"
 
+#include <mutex>
+
 #include <cuda.h>
 
 namespace tman {
@@ -994,7 +996,9 @@ inline bool gemm_pair(int M) { return M > BM; }
 // writes about 50 GB/s; the more pieces per tile, the more to read back).
 struct GemmPlan { int pair, mh, tiles_m, tiles_n, span_tiles, workers, col_fastest, split_s; };
 
-GemmPlan plan_gemm(int M, int K, int N, int bits, int sms)
+// `resident`: how many workers (CTAs, or CTA pairs) of the chosen kernel the device can hold at the
+// same time.  Workers wait for one another's partial tiles, so no more than that may be launched.
+GemmPlan plan_gemm(int M, int K, int N, int bits, int sms, int resident)
 {
     GemmPlan g;
     g.pair = gemm_pair(M) ? 1 : 0;
@@ -1003,6 +1007,7 @@ GemmPlan plan_gemm(int M, int K, int N, int bits, int sms)
     g.tiles_m = (M + rows - 1) / rows;
     const long long nu = K / (2 * BK);
     long long workers = (sms < kMaxGemmCtas ? sms : kMaxGemmCtas) / ncta;
+    if (workers > resident) workers = resident;
     if (workers < 1) workers = 1;
     const int n32 = (N + 31) / 32, tn_min = (n32 + BN / 32 - 1) / (BN / 32);
     const bool pair = g.pair != 0;
@@ -1103,16 +1108,68 @@ tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, co
     return launch_cfg<BITS, 2, true>(tmap_x, tmap_w, tmap_y, p, g.workers, s);
 }
 
+// Workers of one kernel variant that can be resident together on the current device (occupancy query,
+// once per device and variant).
+template <int BITS, int MH, bool PAIR>
+int resident_cfg(int sms)
+{
+    using C = Cfg<MH, PAIR>;
+    auto kern = mpgemm_kernel<BITS, MH, PAIR>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes(BITS)) != cudaSuccess) return -1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(sms / C::NCTA * C::NCTA));
+    cfg.blockDim = dim3(GEMM_THREADS);
+    cfg.dynamicSmemBytes = C::smem_bytes(BITS);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C::NCTA;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) return -1;
+    return n;
+}
+
+int resident_workers(int M, int bits, int sms)
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex lock;
+    static int cache[kMaxDevices][3][3];     // [device][bits - 2][variant], 0 = not asked yet
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices || bits < 2 || bits > 4) return -1;
+    const int variant = !gemm_pair(M) ? 0 : (gemm_mh(M) == 1 ? 1 : 2);
+    std::lock_guard<std::mutex> guard(lock);
+    int &slot = cache[dev][bits - 2][variant];
+    if (slot == 0) {
+        int n = -1;
+        if (bits == 2) n = variant == 0 ? resident_cfg<2, 1, false>(sms) : variant == 1 ? resident_cfg<2, 1, true>(sms) : resident_cfg<2, 2, true>(sms);
+        if (bits == 3) n = variant == 0 ? resident_cfg<3, 1, false>(sms) : variant == 1 ? resident_cfg<3, 1, true>(sms) : resident_cfg<3, 2, true>(sms);
+        if (bits == 4) n = variant == 0 ? resident_cfg<4, 1, false>(sms) : variant == 1 ? resident_cfg<4, 1, true>(sms) : resident_cfg<4, 2, true>(sms);
+        if (n < 1) return -1;                 // not cached: asked again next time
+        slot = n;
+    }
+    return slot;
+}
+
 }  // namespace
 
-tman_status mpgemm_plan(int M, int K, int N, int *out8)
+tman_status mpgemm_plan_for(int M, int K, int N, int bits, int sms, int resident, int *out8)
 {
-    const int sms = sm_count();
-    if (sms <= 0) return TMAN_ERR_CUDA;
-    const GemmPlan g = plan_gemm(M, K, N, 4, sms);
+    const GemmPlan g = plan_gemm(M, K, N, bits, sms, resident);
     out8[0] = g.pair; out8[1] = g.mh; out8[2] = g.tiles_m; out8[3] = g.tiles_n; out8[4] = (g.span_tiles || g.split_s) ? 0 : 1; out8[5] = g.workers;
     out8[6] = g.span_tiles; out8[7] = g.split_s;
     return TMAN_OK;
+}
+
+tman_status mpgemm_plan(int M, int K, int N, int bits, int *out8)
+{
+    const int sms = sm_count();
+    if (sms <= 0) return TMAN_ERR_CUDA;
+    const int resident = resident_workers(M, bits, sms);
+    if (resident < 1) return TMAN_ERR_CUDA;
+    return mpgemm_plan_for(M, K, N, bits, sms, resident, out8);
 }
 
 size_t mpgemm_workspace_bytes(int M, int, int)
@@ -1129,7 +1186,9 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     if (!enc) return TMAN_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
-    const GemmPlan g = plan_gemm(M, K, N, bits, sms);
+    const int resident = resident_workers(M, bits, sms);
+    if (resident < 1) return TMAN_ERR_CUDA;
+    const GemmPlan g = plan_gemm(M, K, N, bits, sms, resident);
     const bool pair = g.pair != 0;
     const int rows_cta = BM * g.mh, bn_cta = pair ? BN / 2 : BN;
     const cuuint32_t estr[3] = {1, 1, 1};

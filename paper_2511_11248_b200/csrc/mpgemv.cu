@@ -34,6 +34,8 @@
 // kernels of the caller's own.
 #include "common.cuh"
 
+#include <atomic>
+
 namespace tman {
 
 constexpr int kGemvThreads = 512;
@@ -698,6 +700,22 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
     auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED, ROLL, HR>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
         return TMAN_ERR_CUDA;
+    // the grid has at most one CTA per SM; the occupancy query says whether an SM can hold one at all
+    // (asked once per device and variant)
+    {
+        constexpr int kMaxDevices = 64;
+        static std::atomic<int> fits[kMaxDevices];          // 0 = not asked, 1 = fits, -1 = does not
+        if (dev < 0 || dev >= kMaxDevices) return TMAN_ERR_CUDA;
+        int f = fits[dev].load(std::memory_order_relaxed);
+        if (f == 0) {
+            int per_sm = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kGemvThreads, kSmem) != cudaSuccess)
+                return TMAN_ERR_CUDA;
+            f = per_sm >= 1 ? 1 : -1;
+            fits[dev].store(f, std::memory_order_relaxed);
+        }
+        if (f < 0) return TMAN_ERR_UNSUPPORTED;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.P, (unsigned)p.nkappa);
     cfg.blockDim = dim3(kGemvThreads);

@@ -101,3 +101,55 @@ def test_workspace_sizes(lib):
     assert B.tman_workspace_bytes(B.OP_GEMM, 1024, 4096, 4096, 4, 128) >= 256
     w = B.tman_workspace_bytes(B.OP_GEMV, 1, 4096, 4096, 4, 64)
     assert w >= 256 + 4096 + 4 * 4096 * 4
+
+
+@pytest.mark.parametrize("offset", [4, 8])
+def test_misaligned_buffers_rejected_before_any_launch(lib, offset):
+    """Packed buffers and workspaces must start on a 256-byte boundary, activations and outputs on a
+    16-byte boundary: every entry point that takes one says TMAN_ERR_SHAPE on the host (the fake
+    pointers are never dereferenced)."""
+    ok = C.c_void_p(4096 * 256)
+    bad = C.c_void_p(4096 * 256 + offset)
+    big = 1 << 30
+    out = C.c_int(0)
+    assert lib.tman_pack_weights(ok, ok, ok, 128, 8, 4, 64, bad, big, None) == 2
+    assert lib.tman_unpack_weights(bad, big, 128, 8, 4, 64, ok, ok, ok, ok, big, None) == 2
+    assert lib.tman_unpack_weights(ok, big, 128, 8, 4, 64, ok, ok, ok, bad, big, None) == 2
+    assert lib.tman_debug_indices(bad, 128, 8, 4, 64, ok, ok, big, None) == 2
+    assert lib.tman_debug_indices(ok, 128, 8, 4, 64, ok, bad, big, None) == 2
+    assert lib.tman_workspace_init(bad, big, None) == 2
+    assert lib.tman_read_status(bad, C.byref(out), None) == 2
+    for fn in (lib.tman_mpgemv, lib.tman_mpgemm):
+        assert fn(bad, big, ok, ok, 1, 128, 8, 4, 64, ok, big, None) == 2      # packed
+        assert fn(ok, big, ok, ok, 1, 128, 8, 4, 64, bad, big, None) == 2      # workspace
+        assert fn(ok, big, bad, ok, 1, 128, 8, 4, 64, ok, big, None) == 2      # activations
+        assert fn(ok, big, ok, bad, 1, 128, 8, 4, 64, ok, big, None) == 2      # output
+    assert lib.tman_mpgemv_static(bad, big, ok, ok, 1, 128, 8, 4, 64, None, None) == 2
+    arr = (C.c_void_p * 1)(bad)
+    good = (C.c_void_p * 1)(ok)
+    sizes = (C.c_size_t * 1)(big)
+    ns = (C.c_int * 1)(8)
+    assert lib.tman_mpgemv_grouped(1, arr, sizes, ok, good, 1, 128, ns, 4, 64, ok, big, None) == 2
+    assert lib.tman_mpgemv_grouped(1, good, sizes, ok, arr, 1, 128, ns, 4, 64, ok, big, None) == 2
+
+
+def test_prefill_plan_never_launches_more_workers_than_can_be_resident(lib):
+    """Workers of a prefill call wait for one another, so the plan is capped by what the device holds
+    at once (the library asks the occupancy query; here the numbers are given).  Host arithmetic only."""
+    from paper_2511_11248_b200 import binding as B
+    shapes = [(1024, 4096, 4096, 4, 128), (1024, 4096, 14336, 4, 128), (8192, 3584, 18944, 2, 64),
+              (100, 24576, 2560, 3, 128), (300, 8192, 1024, 4, 128), (64, 4096, 4096, 4, 64)]
+    for M, K, N, bits, G in shapes:
+        full = B.tman_debug_gemm_plan_for(M, K, N, bits, G, 148, 148)
+        ncta = 2 if full["pair"] else 1
+        assert 1 <= full["workers"] * ncta <= 148
+        for resident in (1, 7, 36, 60):
+            p = B.tman_debug_gemm_plan_for(M, K, N, bits, G, 148, resident)
+            assert 1 <= p["workers"] <= resident, (M, K, N, resident, p)
+            assert p["pair"] == full["pair"] and p["row_blocks"] == full["row_blocks"]
+            # every tile is still covered: whole tiles go round the workers, split tiles have their pieces
+            assert p["tiles_m"] * p["tiles_n"] >= 1
+            if p["pieces"]:
+                assert p["tiles_m"] * p["tiles_n"] * p["pieces"] == p["workers"]
+    with pytest.raises(B.TmanError):
+        B.tman_debug_gemm_plan_for(1024, 4096, 4096, 4, 128, 148, 0)
