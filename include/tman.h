@@ -60,7 +60,9 @@ int tman_version(void);
 tman_status tman_packed_bytes(int K, int N, int bits, int group, size_t *out_bytes /*host*/);
 
 /* Bytes of scratch a call needs.  op: 0 = tman_mpgemv, 1 = tman_mpgemm, 2 = unpack / debug
- * extractors.  The workspace must have been cleared once with tman_workspace_init before its
+ * extractors.  For op 0 the size depends on M: it is what the fastest plan for M rows wants;
+ * tman_mpgemv also accepts any workspace of at least the M = 1 size and then makes more passes over the
+ * weights with fewer rows each (see tman_debug_gemv_plan).  The workspace must have been cleared once with tman_workspace_init before its
  * first use; calls leave it ready for the next call.  Two calls that overlap on the GPU must
  * not share a workspace. */
 tman_status tman_workspace_bytes(int op, int M, int K, int N, int bits, int group,
@@ -203,6 +205,27 @@ tman_status tman_debug_gemm_plan(int M, int K, int N, int bits, int group, int *
  * to launch.  Pure host arithmetic: needs no GPU. */
 tman_status tman_debug_gemm_plan_for(int M, int K, int N, int bits, int group, int sms, int resident,
                                      int *out8 /*host*/);
+
+/* How tman_mpgemv would serve a call of M rows (paper Sec. 4.3 and Sec. 5 "Implementation": the tiling
+ * of the lookup kernel is searched under the hardware's limits; here the searched space is the kernel
+ * variants the library carries).  Host arithmetic only, nothing is launched, needs no GPU.  A variant
+ * carries 1, 2, 4 or 8 activation rows per pass over the weights (table entries of one fp32 row or of
+ * 1, 2 or 4 fp16 row pairs) in K-slices of 16, 32, 16 or 8 plane words.  A variant is admitted when its
+ * K-slices can all be resident (`sms` multiprocessors), its tables fit an SM's shared memory and its
+ * partial sums fit `ws_limit` bytes (0: no limit); among the admitted ones the passes with the least
+ * modelled time (fixed cost per pass + per-megabyte cost of the bit planes, fitted to measurements) are
+ * chosen.  out (host, 52 ints): [0] passes (0: none admissible -> TMAN_ERR_UNSUPPORTED), [1] workspace
+ * KiB the plan needs, [2] modelled time in ns, then six ints per pass from out[4]: rows carried, rows the
+ * variant can carry, plane words per K-slice, K-slices, CTAs launched, shared-memory bytes per CTA. */
+tman_status tman_debug_gemv_plan(int M, int K, int N, int bits, int group, int sms, size_t ws_limit,
+                                 int *out /*host*/);
+
+/* Lets a bounded wait run out, safely: one warp waits, with the same routine the decode kernel's split-K
+ * combine uses, for partial sums that nothing writes (the workspace must be freshly prepared), gives up
+ * after `polls` polls (1 .. 2^20, a few hundred nanoseconds each) and reports TMAN_ERR_TIMEOUT in the
+ * status word like the decode kernel would.  The kernel always ends by itself.  workspace: at least
+ * 256 + 512 bytes.  No counterpart in the paper. */
+tman_status tman_debug_wait_timeout(void *workspace, size_t ws_bytes, unsigned int polls, tman_stream_t stream);
 
 /* Microbenchmarks behind the decode kernel's design, the counterpart on this GPU of the paper's
  * instruction study (Sec. 5 "Implementation", Table 1: lookups per instruction x log2(table entries) =

@@ -23,7 +23,7 @@ EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
     "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
-    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for",
+    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for", "tman_debug_gemv_plan", "tman_debug_wait_timeout",
 ]
 
 _lib = None
@@ -63,6 +63,9 @@ def lib() -> C.CDLL:
         L.tman_debug_gemm_plan.argtypes = [i, i, i, i, i, C.POINTER(C.c_int)]
         L.tman_debug_microbench.argtypes = [i, i, vp, sz, vp, sz, vp]
         L.tman_debug_cluster_capacity.argtypes = [i, i, i, C.POINTER(C.c_int)]
+        L.tman_debug_gemm_plan_for.argtypes = [i, i, i, i, i, i, i, C.POINTER(C.c_int)]
+        L.tman_debug_gemv_plan.argtypes = [i, i, i, i, i, i, sz, C.POINTER(C.c_int)]
+        L.tman_debug_wait_timeout.argtypes = [vp, sz, C.c_uint, vp]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -177,6 +180,19 @@ def tman_debug_gemm_plan_for(M, K, N, bits, group, sms, resident) -> dict:
     out = (C.c_int * 8)()
     _check(lib().tman_debug_gemm_plan_for(M, K, N, bits, group, sms, resident, out), "tman_debug_gemm_plan_for")
     return dict(zip(("pair", "row_blocks", "tiles_m", "tiles_n", "whole_tiles", "workers", "span_tiles", "pieces"), list(out)))
+
+
+def tman_debug_gemv_plan(M, K, N, bits, group, sms=148, ws_limit=0) -> dict:
+    out = (C.c_int * 52)()
+    _check(lib().tman_debug_gemv_plan(M, K, N, bits, group, sms, C.c_size_t(ws_limit), out), "tman_debug_gemv_plan")
+    keys = ("rows", "variant_rows", "words", "slices", "ctas", "smem_bytes")
+    return {"ws_kib": out[1], "cost_us": out[2] / 1000.0,
+            "passes": [dict(zip(keys, out[4 + 6 * i: 10 + 6 * i])) for i in range(out[0])]}
+
+
+def tman_debug_wait_timeout(ws, polls, stream=None) -> None:
+    _check(lib().tman_debug_wait_timeout(_ptr(ws), ws.numel() * ws.element_size(), polls, _stream(stream)),
+           "tman_debug_wait_timeout")
 
 
 def tman_debug_luts(x, M, K, lut, stream=None) -> None:

@@ -48,7 +48,7 @@ tman_status tman_workspace_bytes(int op, int M, int K, int N, int bits, int grou
     if (M < 1) return TMAN_ERR_SHAPE;
     if (op == 0) {
         if (M > 8) return TMAN_ERR_SHAPE;
-        *out_bytes = mpgemv_workspace_bytes(M, K, N);
+        *out_bytes = mpgemv_workspace_bytes(M, K, N, bits);
     } else if (op == 1) {
         *out_bytes = mpgemm_workspace_bytes(M, K, N);
     } else if (op == 2) {
@@ -126,7 +126,7 @@ tman_status tman_mpgemv(const void *packed, size_t packed_bytes, const void *x_f
     tman_status st = check_matmul(packed, packed_bytes, x_f16, y_f16, M, K, N, bits, group, workspace);
     if (st != TMAN_OK) return st;
     if (M > 8) return TMAN_ERR_SHAPE;
-    if (ws_bytes < mpgemv_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (ws_bytes < mpgemv_workspace_bytes(1, K, N, bits)) return TMAN_ERR_BUFFER_TOO_SMALL;
     return launch_mpgemv(packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
                          reinterpret_cast<cudaStream_t>(stream));
 }
@@ -144,7 +144,7 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed, const size
         ntot += N[g];
     }
     if (M > 8 || ntot > (1 << 30)) return TMAN_ERR_SHAPE;
-    if (ws_bytes < mpgemv_workspace_bytes(M, K, (int)ntot)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (ws_bytes < mpgemv_workspace_bytes(1, K, (int)ntot, bits)) return TMAN_ERR_BUFFER_TOO_SMALL;
     return launch_mpgemv_grouped(count, packed, x_f16, y_f16, M, K, N, bits, group, workspace, ws_bytes,
                                  reinterpret_cast<cudaStream_t>(stream));
 }
@@ -197,6 +197,34 @@ tman_status tman_debug_gemm_plan_for(int M, int K, int N, int bits, int group, i
     if (M < 1 || sms < 1 || resident < 1) return TMAN_ERR_SHAPE;
     if (bits < 2) return TMAN_ERR_UNSUPPORTED;
     return mpgemm_plan_for(M, K, N, bits, sms, resident, out8);
+}
+
+tman_status tman_debug_gemv_plan(int M, int K, int N, int bits, int group, int sms, size_t ws_limit, int *out)
+{
+    if (!out) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, bits, group);
+    if (st != TMAN_OK) return st;
+    if (M < 1 || M > kGemvMaxRows || sms < 1) return TMAN_ERR_SHAPE;
+    if (bits < 2) return TMAN_ERR_UNSUPPORTED;
+    const GemvPlan g = plan_gemv(M, K, N, bits, sms, ws_limit ? ws_limit : (size_t)-1);
+    for (int i = 0; i < 4 + 6 * kGemvMaxRows; ++i) out[i] = 0;
+    out[0] = g.npass;
+    out[1] = (int)((g.ws_bytes + 1023) / 1024);
+    out[2] = (int)(g.cost_us * 1000.0 + 0.5);
+    for (int i = 0; i < g.npass; ++i) {
+        int *o = out + 4 + 6 * i;
+        o[0] = g.pass[i].rows; o[1] = g.pass[i].variant_rows; o[2] = g.pass[i].words;
+        o[3] = g.pass[i].nkappa; o[4] = g.pass[i].nkappa * g.pass[i].ctas_per_slice; o[5] = g.pass[i].smem_bytes;
+    }
+    return g.npass ? TMAN_OK : TMAN_ERR_UNSUPPORTED;
+}
+
+tman_status tman_debug_wait_timeout(void *workspace, size_t ws_bytes, unsigned int polls, tman_stream_t stream)
+{
+    if (!workspace) return TMAN_ERR_NULL;
+    if (!aligned_to(workspace, 256)) return TMAN_ERR_SHAPE;
+    if (polls < 1 || polls > (1u << 20)) return TMAN_ERR_SHAPE;
+    return launch_wait_timeout(workspace, ws_bytes, polls, reinterpret_cast<cudaStream_t>(stream));
 }
 
 tman_status tman_debug_microbench(int kind, int arg, void *results, size_t results_bytes, void *buffer,

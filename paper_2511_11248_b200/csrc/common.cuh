@@ -116,7 +116,16 @@ tman_status launch_unpack(const void *packed, int K, int N, int bits, int group,
 tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int group, uint8_t *idx,
                                  uint32_t *status, cudaStream_t s);
 tman_status launch_debug_luts(const void *x, int M, int K, float *lut, cudaStream_t s);
-size_t      mpgemv_workspace_bytes(int M, int K, int N);
+size_t      mpgemv_workspace_bytes(int M, int K, int N, int bits);
+// The decode call's plan: passes over the weights, each with one kernel variant (see mpgemv.cu).
+constexpr int kGemvMaxRows = 8;
+constexpr int kGemvVariantCount = 4;
+constexpr int kGemvSmemLimit = 227 * 1024;
+constexpr int kGemvPlanSms = 148;
+struct GemvPass { int variant, rows, variant_rows, words, nkappa, ctas_per_slice, smem_bytes; };
+struct GemvPlan { int npass; GemvPass pass[kGemvMaxRows]; size_t ws_bytes; double cost_us; };
+tman_status launch_wait_timeout(void *ws, size_t ws_bytes, uint32_t limit, cudaStream_t s);
+GemvPlan    plan_gemv(int M, int K, int N, int bits, int sms, size_t ws_limit);
 tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s);
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                           int group, void *ws, size_t ws_bytes, cudaStream_t s);

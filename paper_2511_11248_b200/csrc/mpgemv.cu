@@ -127,6 +127,25 @@ __device__ __forceinline__ bool has_sentinel(const float4 &v)
            __float_as_uint(v.z) == kGemvSentinel || __float_as_uint(v.w) == kGemvSentinel;
 }
 
+// Bounded wait of the split-K combine: polls up to four partial-sum quads (slices kp, kp + SP, ... below
+// nkappa) until none of them holds the "no sum pending" pattern, at most `limit` times.  Returns
+// whether they all arrived; the caller reports TMAN_ERR_TIMEOUT otherwise.
+__device__ __forceinline__ bool wait_for_sums(const float4 *src, size_t stride4, int kp, int SP, int nkappa,
+                                              uint32_t limit, float4 (&t)[4])
+{
+    bool ready = false;
+    for (uint32_t tries = 0; !ready && tries < limit; ++tries) {
+        ready = true;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (kp + q * SP < nkappa) t[q] = ld_volatile_f4(src + (size_t)(kp + q * SP) * stride4);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (kp + q * SP < nkappa) ready = ready && !has_sentinel(t[q]);
+    }
+    return ready;
+}
+
 // byte offset of table entry (group c of the lane's word, index p, slot) inside the table area
 __device__ __forceinline__ constexpr uint32_t table_imm(int c) { return (uint32_t)(c >> 1) * 65536u + (uint32_t)(c & 1) * 128u; }
 
@@ -630,17 +649,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int kp = part; alive && kp < p.nkappa; kp += 4 * SP) {
                 float4 t[4];
-                bool ready = false;
-                for (uint32_t tries = 0; !ready && tries < kGemvPollLimit; ++tries) {
-                    ready = true;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        if (kp + q * SP < p.nkappa) t[q] = ld_volatile_f4(src + (size_t)(kp + q * SP) * stride4);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        if (kp + q * SP < p.nkappa) ready = ready && !has_sentinel(t[q]);
-                }
-                if (!ready) { gave_up = true; break; }
+                if (!wait_for_sums(src, stride4, kp, SP, p.nkappa, kGemvPollLimit, t)) { gave_up = true; break; }
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     if (kp + q * SP < p.nkappa) {
@@ -737,32 +746,101 @@ static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
 {
     // one row: fp32 tables over half-warp slices, large units on one rolling set of registers;
     // more rows: fp16 row pairs, small double-buffered units
-    constexpr int ROLL = HR ? 0 : 1;
-    constexpr int S = HR ? 1 : ((BITS == 2) ? 4 : 2);
+    constexpr int ROLL = (HR && MT == 4) ? 0 : 1;
+    constexpr int S = (HR && MT == 4) ? 1 : (HR && MT == 2) ? 2 : ((BITS == 2) ? 4 : 2);
     constexpr int HALF = HR ? 0 : 1;
     if (p.count > 1) return launch_one<BITS, MT, S, PRE, HALF, 1, ROLL, HR>(p, sms, s);
     return launch_one<BITS, MT, S, PRE, HALF, 0, ROLL, HR>(p, sms, s);
 }
 
-// Rows a launch carries and plane words per K-slice, by the number of rows in the call: 1 row -> fp32
-// tables, 16 words; 2 rows -> one fp16 pair per entry, 32 words; 3-4 rows -> two pairs, 16 words;
-// 5-8 rows -> four pairs, 8 words.
-static void gemv_variant(int M, int *rows, int *words)
+// ---- the plan: which kernel variants serve a call (host arithmetic only) -------------------------
+// A variant carries up to `rows` activation rows per pass over the weights in K-slices of `words` plane
+// words; its table entries have `slots` 32-bit slots (one fp32 row, or two fp16 rows each).  The time of a
+// pass is modelled as fixed + per_mb x megabytes of bit planes; the constants were fitted to calls timed
+// in a CUDA graph on a B200 (K = 4096, N = 14336; 2- and 4-bit for one row, 4-bit for the others):
+//   rows 1: 6.9 / 9.7 us   rows 2: 11.4 us   rows 4: 15.3 us   rows 8: 25.6 us.
+// The slope grows with the rows because an entry of 2 / 4 / 8 fp16 rows takes 1 / 2 / 4 shared-memory
+// wavefronts per lookup.
+struct GemvVariant { int rows, words, slots, half_slices; double fixed_us, us_per_mb; };
+static const GemvVariant kGemvVariants[kGemvVariantCount] = {
+    {1, 16, 1, 1, 4.10, 0.190},
+    {2, 32, 1, 0, 4.35, 0.240},
+    {4, 16, 2, 0, 4.85, 0.355},
+    {8, 8, 4, 0, 5.85, 0.670},
+};
+
+static size_t variant_ws_bytes(const GemvVariant &v, int K, int N)
 {
-    if (M <= 1) { *rows = 1; *words = 16; }
-    else if (M == 2) { *rows = 2; *words = 32; }
-    else if (M <= 4) { *rows = 4; *words = 16; }
-    else { *rows = 8; *words = 8; }
+    // one fp32 partial sum per K-slice, row of the variant and column
+    const size_t nkappa = (size_t)(K / 32 + v.words - 1) / (size_t)v.words;
+    return kWsStatusBytes + nkappa * (size_t)v.rows * (size_t)N * sizeof(float);
+}
+
+// Limits a variant must meet on this device and call: its K-slices times at least one CTA each must be
+// resident together (the CTAs poll one another's partial sums), its tables must fit the shared memory of
+// an SM, and its partial sums must fit the caller's workspace.
+static bool variant_feasible(const GemvVariant &v, int K, int N, int sms, size_t ws_limit)
+{
+    const int nkappa = (K / 32 + v.words - 1) / v.words;
+    const int smem = (v.half_slices ? kGemvTableBytes / 2 : kGemvTableBytes) + 64;
+    return nkappa <= sms && smem <= kGemvSmemLimit && variant_ws_bytes(v, K, N) <= ws_limit;
+}
+
+GemvPlan plan_gemv(int M, int K, int N, int bits, int sms, size_t ws_limit)
+{
+    // best[m]: least modelled time for m rows; a pass with variant v takes min(rows_v, m) of them
+    const double plane_mb = (double)K * (double)N * bits / 8.0 / 1e6;
+    double best[kGemvMaxRows + 1];
+    int pick[kGemvMaxRows + 1];
+    for (int m = 0; m <= kGemvMaxRows; ++m) { best[m] = 1e300; pick[m] = -1; }
+    best[0] = 0.0;
+    for (int m = 1; m <= M && m <= kGemvMaxRows; ++m) {
+        best[m] = 1e300;
+        pick[m] = -1;
+        for (int vi = 0; vi < kGemvVariantCount; ++vi) {
+            const GemvVariant &v = kGemvVariants[vi];
+            if (!variant_feasible(v, K, N, sms, ws_limit)) continue;
+            const int take = v.rows < m ? v.rows : m;
+            if (take < v.rows && vi > 0 && kGemvVariants[vi - 1].rows >= take &&
+                variant_feasible(kGemvVariants[vi - 1], K, N, sms, ws_limit))
+                continue;                                   // a narrower variant carries these rows as well
+            const double c = v.fixed_us + v.us_per_mb * plane_mb + best[m - take];
+            if (c < best[m] - 1e-9) { best[m] = c; pick[m] = vi; }
+        }
+        if (pick[m] < 0) break;
+    }
+    GemvPlan g = {};
+    if (M < 1 || M > kGemvMaxRows || pick[M] < 0) return g;      // npass == 0: no feasible plan
+    g.cost_us = best[M];
+    // widest passes first
+    int left = M;
+    while (left > 0) {
+        const int vi = pick[left];
+        const GemvVariant &v = kGemvVariants[vi];
+        const int take = v.rows < left ? v.rows : left;
+        GemvPass &ps = g.pass[g.npass++];
+        ps.variant = vi;
+        ps.rows = take;
+        ps.variant_rows = v.rows;
+        ps.words = v.words;
+        ps.nkappa = (K / 32 + v.words - 1) / v.words;
+        ps.ctas_per_slice = sms / ps.nkappa;
+        ps.smem_bytes = v.half_slices ? kGemvTableBytes / 2 : kGemvTableBytes + 64;
+        const size_t need = variant_ws_bytes(v, K, N);
+        if (need > g.ws_bytes) g.ws_bytes = need;
+        left -= take;
+    }
+    return g;
 }
 
 template <int BITS>
-static tman_status launch_rows(GemvParams p, int rows, int sms, cudaStream_t s)
+static tman_status launch_rows(GemvParams p, int rows, int variant, int sms, cudaStream_t s)
 {
     p.M = rows;
     const bool pre = p.group >= 64;
-    if (rows == 1) return pre ? launch_mt<BITS, 1, 1, 0>(p, sms, s) : launch_mt<BITS, 1, 0, 0>(p, sms, s);
-    if (rows == 2) return pre ? launch_mt<BITS, 1, 1, 1>(p, sms, s) : launch_mt<BITS, 1, 0, 1>(p, sms, s);
-    if (rows <= 4) return pre ? launch_mt<BITS, 2, 1, 1>(p, sms, s) : launch_mt<BITS, 2, 0, 1>(p, sms, s);
+    if (variant == 0) return pre ? launch_mt<BITS, 1, 1, 0>(p, sms, s) : launch_mt<BITS, 1, 0, 0>(p, sms, s);
+    if (variant == 1) return pre ? launch_mt<BITS, 1, 1, 1>(p, sms, s) : launch_mt<BITS, 1, 0, 1>(p, sms, s);
+    if (variant == 2) return pre ? launch_mt<BITS, 2, 1, 1>(p, sms, s) : launch_mt<BITS, 2, 0, 1>(p, sms, s);
     return pre ? launch_mt<BITS, 4, 1, 1>(p, sms, s) : launch_mt<BITS, 4, 0, 1>(p, sms, s);
 }
 
@@ -770,6 +848,25 @@ __global__ void ws_fill_kernel(uint32_t *ws, size_t words)
 {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < words) ws[i] = (i < kWsStatusBytes / 4) ? 0u : kGemvSentinel;
+}
+
+// One CTA waits, with the combine's own bounded wait, for partial sums that nothing will ever write (the
+// workspace holds "no sum pending" after tman_workspace_init), gives up after `limit` polls and reports
+// it the way the decode kernel does.  For testing that a wait that runs out ends cleanly.
+__global__ void wait_timeout_kernel(float *partials, uint32_t *status, uint32_t limit)
+{
+    float4 t[4];
+    const bool ready = wait_for_sums(reinterpret_cast<const float4 *>(partials) + threadIdx.x, 0, 0, 1, 1, limit, t);
+    const bool gave_up = __any_sync(0xffffffffu, !ready);
+    if (gave_up && threadIdx.x == 0) atomicCAS(status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
+}
+
+tman_status launch_wait_timeout(void *ws, size_t ws_bytes, uint32_t limit, cudaStream_t s)
+{
+    if (ws_bytes < kWsStatusBytes + 32 * sizeof(float4)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    uint8_t *w8 = static_cast<uint8_t *>(ws);
+    wait_timeout_kernel<<<1, 32, 0, s>>>(reinterpret_cast<float *>(w8 + kWsStatusBytes), reinterpret_cast<uint32_t *>(w8), limit);
+    return launch_status();
 }
 
 // status word (and its padding) zero, everything after it "no sum pending"
@@ -780,21 +877,24 @@ tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s)
     return launch_status();
 }
 
-size_t mpgemv_workspace_bytes(int M, int K, int N)
+size_t mpgemv_workspace_bytes(int M, int K, int N, int bits)
 {
-    // one fp32 partial sum per K-slice, row of the launch and column
-    int rows = 1, words = 16;
-    gemv_variant(M, &rows, &words);
-    const size_t nkappa = (size_t)(K / 32 + words - 1) / (size_t)words;
-    return kWsStatusBytes + nkappa * (size_t)rows * (size_t)N * sizeof(float);
+    // what the preferred plan needs (on the reference device size: the choice of variants depends on the
+    // SM count only through the limit on K-slices); a smaller workspace makes the call fall back to
+    // variants with fewer rows per pass, down to what one row needs
+    const GemvPlan g = plan_gemv(M, K, N, bits, kGemvPlanSms, (size_t)-1);
+    return g.npass ? g.ws_bytes : (size_t)-1;
 }
 
 tman_status launch_mpgemv_grouped(int count, const void *const *packed, const void *x, void *const *y, int M, int K,
                                   const int *Ns, int bits, int group, void *ws, size_t ws_bytes, cudaStream_t s)
 {
-    (void)ws_bytes;
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
+    int ntot = 0;
+    for (int g = 0; g < count; ++g) ntot += Ns[g];
+    const GemvPlan plan = plan_gemv(M, K, ntot, bits, sms, ws_bytes);
+    if (plan.npass == 0) return TMAN_ERR_UNSUPPORTED;
     uint8_t *w8 = static_cast<uint8_t *>(ws);
     GemvParams p;
     p.count = count;
@@ -818,17 +918,19 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
     p.M = 0; p.nkappa = 0; p.P = 0; p.units = 0;
     p.group_shift = (group == 32) ? 5 : (group == 64) ? 6 : 7;
     p.nblk = K / group;
-    // a table entry carries up to eight rows (four fp16 pairs): one pass over the weights for M <= 8
-    for (int m0 = 0; m0 < M; m0 += 8) {
-        const int rows = (M - m0 < 8) ? (M - m0) : 8;
+    // a table entry carries up to eight rows (four fp16 pairs): normally one pass over the weights
+    int m0 = 0;
+    for (int ps = 0; ps < plan.npass; ++ps) {
+        const int rows = plan.pass[ps].rows, variant = plan.pass[ps].variant;
         p.x = static_cast<const __half *>(x) + (size_t)m0 * K;
         for (int g = 0; g < kGemvMaxGroup; ++g)
             p.y[g] = static_cast<__half *>(y[g < count ? g : 0]) + (size_t)m0 * p.Ng[g];
         tman_status st;
-        if (bits == 2) st = launch_rows<2>(p, rows, sms, s);
-        else if (bits == 3) st = launch_rows<3>(p, rows, sms, s);
-        else st = launch_rows<4>(p, rows, sms, s);
+        if (bits == 2) st = launch_rows<2>(p, rows, variant, sms, s);
+        else if (bits == 3) st = launch_rows<3>(p, rows, variant, sms, s);
+        else st = launch_rows<4>(p, rows, variant, sms, s);
         if (st != TMAN_OK) return st;
+        m0 += rows;
     }
     return TMAN_OK;
 }

@@ -62,7 +62,7 @@ extern "C" tman_status tman_mpgemv_static(const void *packed, size_t packed_byte
         (reinterpret_cast<uintptr_t>(y_f16) & 15))
         return TMAN_ERR_SHAPE;
     // the fixed array is the whole budget: a shape whose scratch does not fit is refused
-    const size_t need = mpgemv_workspace_bytes(M, K, N);
+    const size_t need = mpgemv_workspace_bytes(M, K, N, bits);
     if (need > kStaticWsBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
 
     void *ws = nullptr;

@@ -35,6 +35,9 @@ def test_library_exports_every_declared_symbol(lib):
     assert set(binding.EXPORTS) <= names
     for n in names:
         assert hasattr(binding, n), f"binding lacks {n}"
+    # every entry point has its argument types declared: ctypes would otherwise pass pointers as 32-bit ints
+    for n in names - {"tman_version"}:
+        assert getattr(lib, n).argtypes is not None, f"{n} has no argtypes"
 
 
 def test_version_and_status_strings(lib):
@@ -153,3 +156,42 @@ def test_prefill_plan_never_launches_more_workers_than_can_be_resident(lib):
                 assert p["tiles_m"] * p["tiles_n"] * p["pieces"] == p["workers"]
     with pytest.raises(B.TmanError):
         B.tman_debug_gemm_plan_for(1024, 4096, 4096, 4, 128, 148, 0)
+
+
+def test_decode_plan_choices_and_limits(lib):
+    """The decode plan (host arithmetic): one pass for every M on the model shapes, fewer rows per pass
+    when the workspace or the number of SMs does not admit the wide variants, and every pass within the
+    limits it was admitted under."""
+    from paper_2511_11248_b200 import binding as B
+    K, N, bits, G = 4096, 14336, 4, 128
+    want = {1: [1], 2: [2], 3: [4], 4: [4], 6: [8], 7: [8], 8: [8]}
+    for M, variants in want.items():
+        p = B.tman_debug_gemv_plan(M, K, N, bits, G)
+        assert [q["variant_rows"] for q in p["passes"]] == variants, (M, p)
+        assert sum(q["rows"] for q in p["passes"]) == M
+        assert p["ws_kib"] * 1024 >= B.tman_workspace_bytes(B.OP_GEMV, M, K, N, bits, G) > (p["ws_kib"] - 1) * 1024
+        for q in p["passes"]:
+            assert q["ctas"] <= 148 and q["slices"] * q["words"] * 32 >= K
+            assert q["smem_bytes"] <= 227 * 1024
+    # five rows: one 8-row pass or a 4-row and a 1-row pass, whichever the model says; all rows served
+    p5 = B.tman_debug_gemv_plan(5, K, N, bits, G)
+    assert sum(q["rows"] for q in p5["passes"]) == 5 and len(p5["passes"]) <= 2
+    # a workspace that only holds the 4-row variant's partial sums: eight rows go in two passes of four
+    ws4 = B.tman_workspace_bytes(B.OP_GEMV, 4, K, N, bits, G)
+    p = B.tman_debug_gemv_plan(8, K, N, bits, G, ws_limit=ws4)
+    assert [q["variant_rows"] for q in p["passes"]] == [4, 4] and p["ws_kib"] * 1024 <= ws4 + 1023
+    # the smallest workspace the call accepts: single rows
+    ws1 = B.tman_workspace_bytes(B.OP_GEMV, 1, K, N, bits, G)
+    p = B.tman_debug_gemv_plan(3, K, N, bits, G, ws_limit=ws1)
+    assert all(q["variant_rows"] <= 2 for q in p["passes"]) and sum(q["rows"] for q in p["passes"]) == 3
+    with pytest.raises(B.TmanError) as e:
+        B.tman_debug_gemv_plan(3, K, N, bits, G, ws_limit=ws1 - 1024)
+    assert e.value.status == 3
+    # a long reduction on a small device: the 8-word K-slices would need more CTAs than there are SMs
+    p = B.tman_debug_gemv_plan(8, 16384, 4096, 2, 64, sms=40)
+    assert all(q["slices"] <= 40 for q in p["passes"]) and sum(q["rows"] for q in p["passes"]) == 8
+    assert all(q["variant_rows"] < 8 for q in p["passes"])
+    # more rows never cost less, more bits never cost less
+    costs = [B.tman_debug_gemv_plan(M, K, N, bits, G)["cost_us"] for M in range(1, 9)]
+    assert all(a <= b + 1e-9 for a, b in zip(costs, costs[1:]))
+    assert B.tman_debug_gemv_plan(4, K, N, 2, G)["cost_us"] < B.tman_debug_gemv_plan(4, K, N, 4, G)["cost_us"]

@@ -64,6 +64,41 @@ def test_pack_directly_followed_by_decode_on_one_stream():
         assert np.array_equal(H.to_f64(y), want)
 
 
+@pytest.mark.parametrize("M,rows_ws", [(8, 4), (8, 1), (3, 1), (5, 2)])
+def test_smaller_workspace_means_more_passes_and_the_same_answer(M, rows_ws):
+    # a workspace sized for fewer rows is accepted; the call then makes several passes over the weights
+    K, N, bits, G = 2048, 264, 4, 64
+    c = synth.small_case(M, K, N, bits, G, seed=60 + M)
+    dev = H.device_case(c)
+    packed = H.pack_case(c, dev)
+    nbytes = B.tman_workspace_bytes(B.OP_GEMV, rows_ws, K, N, bits, G)
+    plan = B.tman_debug_gemv_plan(M, K, N, bits, G, ws_limit=nbytes)
+    assert len(plan["passes"]) >= 2
+    ws = H.guarded_bytes(nbytes, "small workspace")
+    B.tman_workspace_init(ws)
+    y = H.alloc_y(M, N)
+    B.tman_mpgemv(packed, dev["x"], y, M, K, N, bits, G, ws)
+    assert B.tman_read_status(ws) == 0
+    H.check_guards()
+    ref = orc.mpgemm(c.x, c.codes, c.scales, c.zeros, c.group)
+    assert rel_err(H.to_f64(y), ref) <= TOL
+
+
+def test_a_wait_that_runs_out_ends_cleanly_with_status_timeout():
+    # nothing ever writes the sums the kernel waits for: it must give up by itself and say so
+    ws = H.alloc_workspace(B.OP_GEMV, 1, 4096, 4096, 2, 64)
+    B.tman_debug_wait_timeout(ws, 2000)
+    assert B.tman_read_status(ws) == 7          # TMAN_ERR_TIMEOUT
+    # the context is intact and the workspace, prepared again, serves a real call
+    B.tman_workspace_init(ws)
+    c = synth.small_case(1, 1024, 32, 2, 64, seed=91)
+    dev = H.device_case(c)
+    y = H.alloc_y(1, 32)
+    B.tman_mpgemv(H.pack_case(c, dev), dev["x"], y, 1, 1024, 32, 2, 64, ws)
+    assert B.tman_read_status(ws) == 0
+    assert rel_err(H.to_f64(y), orc.mpgemm(c.x, c.codes, c.scales, c.zeros, c.group)) <= TOL
+
+
 def test_repeat_calls_share_workspace_and_agree():
     c = synth.small_case(2, 2048, 264, 4, 64, seed=21)
     dev = H.device_case(c)
