@@ -442,12 +442,12 @@ def run_ours(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
-# profiles/.  mpGEMV: one gate/up-sized launch moved 17.04 MB for 16.78 MB of algorithmic bytes
-# (+1.55 %); traffic grows with the bytes streamed, so the step's mean launch (25.17 MB) is scaled
-# by the same ratio.  mpGEMM: none (the kernel has changed since its counters were taken: 41.6 MB for
-# the M=1024, K=4096, N=14336 launch at that time).
-TRAFFIC_BYTES_PER_LAUNCH = 25171968.0 * (17.04 / 16.78)
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+# profiles/.  mpGEMV: one gate/up-sized launch moved 17.03 MB for 16.78 MB of algorithmic bytes
+# (+1.5 %); traffic grows with the bytes streamed, so the step's mean launch (25.17 MB) is scaled
+# by the same ratio.  mpGEMM: the M=1024, K=4096, N=14336 launch (the larger of the two timed shapes)
+# read 39.2 MB and wrote 0.4 - 2.5 MB (the output mostly stays in L2).
+TRAFFIC_BYTES_PER_LAUNCH = 25171968.0 * (17.03 / 16.78)
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 40.6e6
 
 
 # Warp instructions the decode kernel executes for one gate/up-sized launch (16.78 MB of algorithmic
@@ -518,6 +518,7 @@ def bench_gemm(torch, B, H, synth, peaks):
                             "(sum of flops / sum of time; 4 rotating copies of inputs and outputs, 40 calls each)",
                 "achieved": tf, "peak": peaks["tf_burst"], "unit": "TFLOP/s", "frac": tf / peaks["tf_burst"],
                 "frac_of_nominal_fp16": tf / NOMINAL_FP16_TFLOPS, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
+                "traffic_of": "the M=1024, K=4096, N=14336 launch",
                 "peak_source": f"of {peaks['src']} (bf16 burst; fp16 has the same nominal rate)"})
     return out
 
