@@ -4,6 +4,7 @@
     python bench.py --leg config1                  # decode, M=1, 4096x4096, 4-bit, group 64
     python bench.py --leg config3 [--dense]        # one decoder layer's projections, bits {2,3,4} x M {1,2,4,8}
     python bench.py --leg config5 [--dense] [--all-groups]   # prefill shapes, M in {128,512,2048,8192}
+    python bench.py --leg ablation                 # prefill with ConvertDQ / LoadFull / sequential in place of the product path
     python bench.py --leg microbench               # lookup rates, load paths, cluster exchange
 
 Everything goes through the C ABI; one JSON line per result on stdout.  Weights and activations are
@@ -42,9 +43,10 @@ def event_us(torch, fn, reps):
     return float(np.median(ts)), float(np.min(ts))
 
 
-def device_problem(torch, B, H, M, K, N, bits, group, seed):
+def device_problem(torch, B, H, M, K, N, bits, group, seed, with_fp16_weights=False):
     """Seeded synthetic weights (uniform codes and zero-points, scales in [0.005, 0.02]) packed by the
-    library, and activations ~ N(0, 1), all drawn on the device."""
+    library, and activations ~ N(0, 1), all drawn on the device.  with_fp16_weights: also the dequantized
+    weights as fp16 [N][K] (what the LoadFull ablation variant reads)."""
     g = torch.Generator(device="cuda")
     g.manual_seed(seed)
     codes = torch.randint(0, 1 << bits, (K, N), dtype=torch.uint8, device="cuda", generator=g)
@@ -53,6 +55,9 @@ def device_problem(torch, B, H, M, K, N, bits, group, seed):
     x = torch.randn((M, K), device="cuda", generator=g).to(torch.float16)
     packed = torch.empty(B.tman_packed_bytes(K, N, bits, group), dtype=torch.uint8, device="cuda")
     B.tman_pack_weights(codes, scales, zeros, K, N, bits, group, packed)
+    if with_fp16_weights:
+        w = scales.float().repeat_interleave(group, 0) * (codes.float() - zeros.float().repeat_interleave(group, 0))
+        return packed, x, w.to(torch.float16).t().contiguous()
     return packed, x
 
 
@@ -291,6 +296,52 @@ def config5(args, rest=()):
     ap.add_argument("--reps", type=int, default=7)
     a = ap.parse_args(list(rest))
     for r in config5_results(torch, B, H, a.reps, a.dense, groups=(64, 128) if a.all_groups else (128,)):
+        print(json.dumps(r), flush=True)
+
+
+# ---- ablations (paper Sec. 6.5) --------------------------------------------------------------------------
+
+ABLATION_SHAPES = [(128, 4096, 4096), (1024, 4096, 4096), (1024, 4096, 14336), (4096, 4096, 14336)]
+
+
+def ablation_results(torch, B, H, reps=7, shapes=ABLATION_SHAPES, group=128):
+    """4-bit prefill with one part replaced: ConvertDQ and LoadFull against the lookup dequantization,
+    sequential against pipelined; LoadFull is also the kernel's own fp16 GEMM (no dequantization at all),
+    so product / load_full is the overhead of fusing the dequantization.  torch.matmul with fp16 weights
+    is the library yardstick."""
+    out = []
+    for M, K, N in shapes:
+        p0, x, wt0 = device_problem(torch, B, H, M, K, N, 4, group, seed=9, with_fp16_weights=True)
+        ncopy = max(2, int(2.2 * L2_BYTES // wt0.numel() // 2) + 1)
+        pk = [p0] + [p0.clone() for _ in range(ncopy - 1)]
+        wts = [wt0] + [wt0.clone() for _ in range(ncopy - 1)]
+        ws = workspace(torch, B, B.OP_GEMM, M, K, N, 4, group)
+        ys = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in range(2)]
+        row = {"leg": "ablation", "M": M, "K": K, "N": N, "bits": 4, "group": group, "copies": ncopy}
+        for name in ("product", "convert_dq", "load_full", "sequential"):
+            def run():
+                for i in range(ncopy):
+                    B.tman_debug_mpgemm_variant(name, pk[i], x, ys[i % 2], M, K, N, 4, group, ws, wts[i])
+            run()
+            torch.cuda.synchronize()
+            row[name + "_us"] = round(event_us(torch, run, reps)[0] / ncopy, 1)
+        assert B.tman_read_status(ws) == 0
+        del pk, wts
+        torch.cuda.empty_cache()
+        row["dense_fp16_torch_us"] = round(dense_case_us(torch, M, K, N, reps), 1)
+        row["convert_dq_over_product"] = round(row["convert_dq_us"] / row["product_us"], 2)
+        row["sequential_over_product"] = round(row["sequential_us"] / row["product_us"], 2)
+        row["product_over_load_full"] = round(row["product_us"] / row["load_full_us"], 2)
+        row["product_TFLOPs"] = round(2.0 * M * K * N / row["product_us"] / 1e6, 1)
+        out.append(row)
+        torch.cuda.empty_cache()
+    return out
+
+
+def ablation(args, rest=()):
+    import torch
+    from paper_2511_11248_b200 import binding as B, helpers as H
+    for r in ablation_results(torch, B, H):
         print(json.dumps(r), flush=True)
 
 

@@ -190,6 +190,24 @@ tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int g
  * device routine the decode kernel builds its tables from (paper Sec. 2.2). */
 tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_stream_t stream);
 
+/* tman_mpgemm with one part of the method replaced, for the ablations of paper Sec. 6.5 ("Efficiency of
+ * the LUT-dequant kernel": against converting with floating-point instructions and against loading
+ * full-precision weights; "Gain from pipelined execution": against doing load, dequantization and
+ * multiplication in turn).  Every variant returns the same y as tman_mpgemm (same bits); only the time
+ * differs.  Arguments as tman_mpgemm, plus
+ *   variant 0  the product path (two-level lookup dequantization, pipelined)
+ *           1  ConvertDQ: every code converted to fp16 with an integer-to-float instruction, zero-point
+ *              subtracted, scale multiplied
+ *           2  LoadFull: no dequantization; fp16 weights wt_f16 [N][K] (device, 16-byte aligned, row n =
+ *              fp16(s * (q - z)) of channel n) are loaded by TMA in place of the packed tiles
+ *           3  Sequential: the product's dequantization with a ring of one stage, so that the load, the
+ *              dequantization and the multiplication of a k-block follow one another
+ *   wt_f16  used by variant 2 only (else may be NULL).
+ * Variants 1-3 exist for bits == 4 (TMAN_ERR_UNSUPPORTED otherwise). */
+tman_status tman_debug_mpgemm_variant(int variant, const void *packed, size_t packed_bytes, const void *x_f16,
+                                      void *y_f16, int M, int K, int N, int bits, int group, const void *wt_f16,
+                                      void *workspace, size_t ws_bytes, tman_stream_t stream);
+
 /* How tman_mpgemm would cut a call's work on the current device (host-side decision, nothing is
  * launched; no counterpart in the paper).  out8 (host) receives: 1 if pairs of CTAs work on a tile
  * else 0; 128-token row blocks per CTA; row tiles; column tiles; 1 if every tile is dealt whole

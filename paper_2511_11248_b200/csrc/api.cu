@@ -160,6 +160,17 @@ tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f
                          reinterpret_cast<cudaStream_t>(stream));
 }
 
+tman_status tman_debug_mpgemm_variant(int variant, const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
+                                      int M, int K, int N, int bits, int group, const void *wt_f16,
+                                      void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    tman_status st = check_matmul(packed, packed_bytes, x_f16, y_f16, M, K, N, bits, group, workspace);
+    if (st != TMAN_OK) return st;
+    if (ws_bytes < mpgemm_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_mpgemm_variant(variant, packed, x_f16, y_f16, M, K, N, bits, group, wt_f16, workspace, ws_bytes,
+                                 reinterpret_cast<cudaStream_t>(stream));
+}
+
 tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int group,
                                uint8_t *idx, void *workspace, size_t ws_bytes, tman_stream_t stream)
 {

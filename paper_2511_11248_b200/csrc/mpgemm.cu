@@ -338,6 +338,38 @@ struct ConvTable {
     }
 };
 
+// Ablation variants of the kernel (paper Sec. 6.5 "Ablation Study"): what replaces the table lookup of the
+// dequantization, or the pipelining.  Every variant computes the same numbers.
+constexpr int kGemmProduct = 0;      // two-level lookup dequantization, pipelined (the product path)
+constexpr int kGemmConvertDq = 1;    // codes converted to floating point one by one, then subtract and multiply
+constexpr int kGemmLoadFull = 2;     // fp16 weights prepared in memory and loaded by TMA, no dequantization
+constexpr int kGemmSequential = 3;   // the product's dequantization with a ring of one stage: load, dequantize, multiply in turn
+
+// The same 32 weights without the conversion table: every code is extracted, converted to fp16 by an
+// integer-to-float conversion, the zero-point subtracted and the scale multiplied (rounds like the table's
+// entries do, so the result is the same bits).
+template <int BITS>
+__device__ __forceinline__ void dequant_word_convert(const uint32_t (&w)[BITS], __half s, uint32_t z, uint32_t (&out)[16])
+{
+    const __half2 s2 = __half2half2(s);
+    const __half2 z2 = __half2half2(__ushort2half_rn((unsigned short)z));
+#pragma unroll
+    for (int ph = 0; ph < 4; ++ph)
+#pragma unroll
+        for (int jp = 0; jp < 4; ++jp) {
+            // weights 8*ph + 2*jp and 8*ph + 2*jp + 1 sit at word bits 4*(2*jp) + ph and 4*(2*jp + 1) + ph
+            uint32_t c0 = 0u, c1 = 0u;
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) {
+                c0 |= ((w[i] >> (8 * jp + ph)) & 1u) << i;
+                c1 |= ((w[i] >> (8 * jp + 4 + ph)) & 1u) << i;
+            }
+            const __half2 c = __halves2half2(__ushort2half_rn((unsigned short)c0), __ushort2half_rn((unsigned short)c1));
+            const __half2 e = __hmul2(s2, __hsub2(c, z2));
+            out[4 * ph + jp] = *reinterpret_cast<const uint32_t *>(&e);
+        }
+}
+
 // 32 weights of one column (one plane word per bit) -> 16 half2 in k order.
 template <int BITS>
 __device__ __forceinline__ void dequant_word(const uint32_t (&w)[BITS], const ConvTable<BITS> &T, uint32_t (&out)[16])
@@ -461,12 +493,13 @@ struct Span {
     }
 };
 
-template <int BITS, int MH, bool PAIR>
+template <int BITS, int MH, bool PAIR, int V>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-              const __grid_constant__ CUtensorMap tmap_y, const GemmParams p)
+              const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_wf, const GemmParams p)
 {
     using C = Cfg<MH, PAIR>;
+    constexpr int RING = (V == kGemmSequential) ? 1 : C::NSTAGE;      // stages of the ring in use
     constexpr int NCTA = C::NCTA, NSTAGE = C::NSTAGE, A_STAGE_BYTES = C::A_STAGE_BYTES, B_STAGE_BYTES = C::B_STAGE_BYTES;
     constexpr int P_PLANE_BYTES = C::P_PLANE_BYTES, P_STAGE_BYTES = BITS * P_PLANE_BYTES, TMEM_COLS = C::TMEM_COLS;
     constexpr int ROWS_CTA = BM * MH;                  // token rows of a tile held by one CTA
@@ -557,15 +590,22 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 const int row0 = tile_rows(sg.tile);
                 const int strip0 = (tile_col0(sg.tile) + (int)rank * (tile_bn(sg.tile) / NCTA)) / 4;
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
-                    const int s = (int)(it % NSTAGE);
-                    const uint32_t ph = (it / NSTAGE) & 1u;
+                    const int s = (int)(it % RING);
+                    const uint32_t ph = (it / RING) & 1u;
                     if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
-                    mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + P_STAGE_BYTES);
-                    tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, row0, loaded0 + 8 * s);
+                    if constexpr (V == kGemmLoadFull) {
+                        // the fp16 weight tile itself: this CTA's channels x one k-block, 128-byte swizzle
+                        mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + B_STAGE_BYTES);
+                        tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, row0, loaded0 + 8 * s);
+                        tma_load_2d(smem_u32(b_tiles + s * B_STAGE_BYTES), &tmap_wf, kb * BK, strip0 * 4, loaded0 + 8 * s);
+                    } else {
+                        mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + P_STAGE_BYTES);
+                        tma_load_2d(smem_u32(a_tiles + s * A_STAGE_BYTES), &tmap_x, kb * BK, row0, loaded0 + 8 * s);
 #pragma unroll
-                    for (int i = 0; i < BITS; ++i)
-                        tma_load_3d(smem_u32(p_tiles + s * P_STAGE_BYTES + i * P_PLANE_BYTES), &tmap_w, kb * (BK / 8), i,
-                                    strip0, loaded0 + 8 * s);
+                        for (int i = 0; i < BITS; ++i)
+                            tma_load_3d(smem_u32(p_tiles + s * P_STAGE_BYTES + i * P_PLANE_BYTES), &tmap_w, kb * (BK / 8), i,
+                                        strip0, loaded0 + 8 * s);
+                    }
                 }
             }
         }
@@ -578,8 +618,8 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tcgen05_fence_after();
                 const uint32_t idesc = (1u << 4) | ((uint32_t)(tile_bn(sg.tile) >> 3) << 17) | ((uint32_t)((NCTA * BM) >> 4) << 24);
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
-                    const int s = (int)(it % NSTAGE);
-                    const uint32_t ph = (it / NSTAGE) & 1u;
+                    const int s = (int)(it % RING);
+                    const uint32_t ph = (it / RING) & 1u;
                     if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
@@ -642,18 +682,20 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             };
             ConvTable<BITS> T;
             int cur_B = -1, next_B = -1;
-            __half sv_next = __float2half(0.f);
-            uint32_t zz_next = 0u;
+            __half sv_next = __float2half(0.f), sv_cur = __float2half(0.f);
+            uint32_t zz_next = 0u, zz_cur = 0u;
             for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
-                const int s = (int)(it % NSTAGE);
-                const uint32_t ph = (it / NSTAGE) & 1u;
-                const bool work = valid && mine(it);
+                const int s = (int)(it % RING);
+                const uint32_t ph = (it / RING) & 1u;
+                const bool work = (V != kGemmLoadFull) && valid && mine(it);
                 if (work) {
                     const int Bk = block_of(kb);
                     if (Bk != cur_B) {
                         if (next_B != Bk) fetch_sz(Bk, sv_next, zz_next);
                         cur_B = Bk;
-                        T.build(sv_next, zz_next);
+                        sv_cur = sv_next;
+                        zz_cur = zz_next;
+                        if constexpr (V != kGemmConvertDq) T.build(sv_next, zz_next);
                     }
                     // scale and zero-point of the block after this one are fetched one k-block ahead
                     const int kn = (ngroup == 1 || !(kb & 1)) ? kb + 1 : kb + 3;
@@ -671,7 +713,8 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     for (int i = 0; i < BITS; ++i)
                         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[i]) : "r"(pp + i * P_PLANE_BYTES) : "memory");
                     uint32_t out[16];
-                    dequant_word<BITS>(w, T, out);
+                    if constexpr (V == kGemmConvertDq) dequant_word_convert<BITS>(w, sv_cur, zz_cur, out);
+                    else dequant_word<BITS>(w, T, out);
                     const uint32_t row = b_base + (uint32_t)s * B_STAGE_BYTES;
 #pragma unroll
                     for (int cj = 0; cj < 4; ++cj) {
@@ -1075,12 +1118,12 @@ GemmPlan plan_gemm(int M, int K, int N, int bits, int sms, int resident)
     return g;
 }
 
-template <int BITS, int MH, bool PAIR>
-tman_status launch_cfg(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const GemmParams &p,
-                       int workers, cudaStream_t s)
+template <int BITS, int MH, bool PAIR, int V>
+tman_status launch_cfg(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const CUtensorMap &tmap_wf,
+                       const GemmParams &p, int workers, cudaStream_t s)
 {
     using C = Cfg<MH, PAIR>;
-    auto kern = mpgemm_kernel<BITS, MH, PAIR>;
+    auto kern = mpgemm_kernel<BITS, MH, PAIR, V>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes(BITS)) != cudaSuccess)
         return TMAN_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -1095,17 +1138,17 @@ tman_status launch_cfg(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, con
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, p) != cudaSuccess) return TMAN_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, tmap_wf, p) != cudaSuccess) return TMAN_ERR_CUDA;
     return TMAN_OK;
 }
 
-template <int BITS>
-tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const GemmParams &p,
-                        const GemmPlan &g, cudaStream_t s)
+template <int BITS, int V>
+tman_status launch_bits(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y, const CUtensorMap &tmap_wf,
+                        const GemmParams &p, const GemmPlan &g, cudaStream_t s)
 {
-    if (!g.pair) return launch_cfg<BITS, 1, false>(tmap_x, tmap_w, tmap_y, p, g.workers, s);
-    if (g.mh == 1) return launch_cfg<BITS, 1, true>(tmap_x, tmap_w, tmap_y, p, g.workers, s);
-    return launch_cfg<BITS, 2, true>(tmap_x, tmap_w, tmap_y, p, g.workers, s);
+    if (!g.pair) return launch_cfg<BITS, 1, false, V>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g.workers, s);
+    if (g.mh == 1) return launch_cfg<BITS, 1, true, V>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g.workers, s);
+    return launch_cfg<BITS, 2, true, V>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g.workers, s);
 }
 
 // Workers of one kernel variant that can be resident together on the current device (occupancy query,
@@ -1114,7 +1157,7 @@ template <int BITS, int MH, bool PAIR>
 int resident_cfg(int sms)
 {
     using C = Cfg<MH, PAIR>;
-    auto kern = mpgemm_kernel<BITS, MH, PAIR>;
+    auto kern = mpgemm_kernel<BITS, MH, PAIR, kGemmProduct>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes(BITS)) != cudaSuccess) return -1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(sms / C::NCTA * C::NCTA));
@@ -1179,8 +1222,19 @@ size_t mpgemm_workspace_bytes(int M, int, int)
 }
 
 tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
-                          int group, void *ws, size_t, cudaStream_t s)
+                          int group, void *ws, size_t ws_bytes, cudaStream_t s)
 {
+    return launch_mpgemm_variant(kGemmProduct, packed, x, y, M, K, N, bits, group, nullptr, ws, ws_bytes, s);
+}
+
+// variant: one of kGemmProduct .. kGemmSequential; wt_f16: for kGemmLoadFull the dequantized weights as fp16
+// [N][K] (channel-major), otherwise unused.  The variants other than the product path exist for 4-bit only.
+tman_status launch_mpgemm_variant(int variant, const void *packed, const void *x, void *y, int M, int K, int N, int bits,
+                                  int group, const void *wt_f16, void *ws, size_t, cudaStream_t s)
+{
+    if (variant < kGemmProduct || variant > kGemmSequential) return TMAN_ERR_UNSUPPORTED;
+    if (variant != kGemmProduct && bits != 4) return TMAN_ERR_UNSUPPORTED;
+    if (variant == kGemmLoadFull && (!wt_f16 || (reinterpret_cast<uintptr_t>(wt_f16) & 15) != 0)) return TMAN_ERR_SHAPE;
     if ((reinterpret_cast<uintptr_t>(x) & 15) != 0 || (reinterpret_cast<uintptr_t>(y) & 15) != 0) return TMAN_ERR_SHAPE;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TMAN_ERR_CUDA;
@@ -1246,9 +1300,24 @@ tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int
     p.span_tiles = g.span_tiles;
     p.split_s = g.split_s;
     p.col_fastest = g.col_fastest;
-    if (bits == 2) return launch_bits<2>(tmap_x, tmap_w, tmap_y, p, g, s);
-    if (bits == 3) return launch_bits<3>(tmap_x, tmap_w, tmap_y, p, g, s);
-    return launch_bits<4>(tmap_x, tmap_w, tmap_y, p, g, s);
+    // the fp16 weights [N][K]: boxes of one k-block x a CTA's channels, 128-byte swizzle (the layout the
+    // dequantization writes); unused maps are copies of the activation map
+    CUtensorMap tmap_wf = tmap_x;
+    if (variant == kGemmLoadFull) {
+        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)bn_cta};
+        if (enc(&tmap_wf, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(wt_f16), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return TMAN_ERR_CUDA;
+    }
+    if (bits == 2) return launch_bits<2, kGemmProduct>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g, s);
+    if (bits == 3) return launch_bits<3, kGemmProduct>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g, s);
+    if (variant == kGemmConvertDq) return launch_bits<4, kGemmConvertDq>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g, s);
+    if (variant == kGemmLoadFull) return launch_bits<4, kGemmLoadFull>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g, s);
+    if (variant == kGemmSequential) return launch_bits<4, kGemmSequential>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g, s);
+    return launch_bits<4, kGemmProduct>(tmap_x, tmap_w, tmap_y, tmap_wf, p, g, s);
 }
 
 }  // namespace tman

@@ -107,6 +107,38 @@ def test_span_cases(M, K, N, bits, G):
     assert torch.equal(y, y2)                       # fixed summation order: same bits
 
 
+def dequantized_fp16_nk(c):
+    """fp16(s * (q - z)) as [N][K]: what the LoadFull variant reads in place of the packed weights."""
+    z = np.repeat(c.zeros.astype(np.float32), c.group, axis=0)
+    s_ = np.repeat(c.scales.astype(np.float32), c.group, axis=0)
+    w = (s_ * (c.codes.astype(np.float32) - z)).astype(np.float16)           # one rounding, like the table's entries
+    return torch.from_numpy(np.ascontiguousarray(w.T).view(np.int16)).cuda().view(torch.float16)
+
+
+@pytest.mark.parametrize("variant", ["convert_dq", "load_full", "sequential"])
+@pytest.mark.parametrize("M,K,N,G", [(100, 384, 136, 128), (600, 512, 7176, 64), (1024, 1024, 3560, 32)])
+def test_ablation_variants_compute_the_same_numbers(variant, M, K, N, G):
+    # Sec. 6.5: the variants replace how fp16 weights come about, or the pipelining; never the result
+    c = synth.small_case(M, K, N, 4, G, seed=M + K + N, outliers=True)
+    dev = H.device_case(c)
+    packed = H.pack_case(c, dev)
+    ws = H.alloc_workspace(B.OP_GEMM, M, K, N, 4, G)
+    want = H.alloc_y(M, N)
+    B.tman_mpgemm(packed, dev["x"], want, M, K, N, 4, G, ws)
+    wt = dequantized_fp16_nk(c) if variant == "load_full" else None
+    got = H.alloc_y(M, N)
+    B.tman_debug_mpgemm_variant(variant, packed, dev["x"], got, M, K, N, 4, G, ws, wt)
+    assert B.tman_read_status(ws) == 0
+    H.check_guards()
+    assert torch.equal(got, want)                     # the same bits as the product path
+    ref = orc.mpgemm(c.x, c.codes, c.scales, c.zeros, c.group)
+    assert rel_err(H.to_f64(got), ref) <= TOL
+    if variant != "load_full":
+        with pytest.raises(B.TmanError) as e:          # the variants exist for 4-bit weights
+            B.tman_debug_mpgemm_variant(variant, packed, dev["x"], got, M, K, N, 2, G, ws, wt)
+        assert e.value.status in (3, 4)
+
+
 def test_integer_case_is_exact():
     rng = np.random.default_rng(5)
     c = synth.small_case(130, 512, 136, 3, 64, seed=31)
