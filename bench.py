@@ -19,7 +19,7 @@ configs 1, 3 and 5 measured in the same run; the end-to-end rate through the C A
 buffers; the CPU oracle's rate on a bounded sample; clocks sampled during the timed region.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-    python bench.py --leg {case,config1,config3,config5,ablation,microbench} [leg options]   # see bench_legs.py
+    python bench.py --leg {case,config1,config3,config5,ablation,ternary,microbench} [leg options]   # see bench_legs.py
 
 With N > 1 (launched under torchrun) every rank runs an independent replica of the same step
 (the path does not shard); value is the sum over ranks divided by the slowest rank's time.
@@ -551,7 +551,7 @@ def main():
     ap.add_argument("--skip-gemm", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-sweeps", action="store_true", help="leave the config 1/3/5 digests out of the line")
-    ap.add_argument("--leg", default="headline", choices=["headline", "case", "config1", "config3", "config5", "ablation", "microbench"],
+    ap.add_argument("--leg", default="headline", choices=["headline", "case", "config1", "config3", "config5", "ablation", "ternary", "microbench"],
                     help="headline: the bench line (default); the others print their own JSON lines")
     args, rest = ap.parse_known_args()
     if args.leg != "headline":

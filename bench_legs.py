@@ -4,6 +4,7 @@
     python bench.py --leg config1                  # decode, M=1, 4096x4096, 4-bit, group 64
     python bench.py --leg config3 [--dense]        # one decoder layer's projections, bits {2,3,4} x M {1,2,4,8}
     python bench.py --leg config5 [--dense] [--all-groups]   # prefill shapes, M in {128,512,2048,8192}
+    python bench.py --leg ternary                  # integer decode: ternary weights, 16-bit integer activations, BitNet sizes
     python bench.py --leg ablation                 # prefill with ConvertDQ / LoadFull / sequential in place of the product path
     python bench.py --leg microbench               # lookup rates, load paths, cluster exchange
 
@@ -296,6 +297,64 @@ def config5(args, rest=()):
     ap.add_argument("--reps", type=int, default=7)
     a = ap.parse_args(list(rest))
     for r in config5_results(torch, B, H, a.reps, a.dense, groups=(64, 128) if a.all_groups else (128,)):
+        print(json.dumps(r), flush=True)
+
+
+# ---- integer path: ternary weights, 16-bit integer activations (paper Sec. 6.1, BitNet kernel sizes) --------
+
+def ternary_results(torch, B, H, reps=7):
+    out = []
+    for K, N in ((2560, 2560), (2560, 6912), (6912, 2560), (6912, 6912)):
+        g = torch.Generator(device="cuda")
+        g.manual_seed(K + N)
+        nbytes = K * N // 4                                   # the bit planes are all the kernel streams
+        ncopy = max(2, int(2.2 * L2_BYTES // nbytes) + 1)
+        group = 128
+        packed = []
+        for _ in range(ncopy):
+            codes = torch.randint(0, 3, (K, N), dtype=torch.uint8, device="cuda", generator=g)
+            pk = torch.empty(B.tman_packed_bytes(K, N, 2, group), dtype=torch.uint8, device="cuda")
+            B.tman_pack_weights(codes, torch.ones((K // group, N), dtype=torch.float16, device="cuda"),
+                                torch.ones((K // group, N), dtype=torch.uint8, device="cuda"), K, N, 2, group, pk)
+            packed.append(pk)
+        x = torch.randn((1, K), device="cuda", generator=g).to(torch.float16)
+        a = torch.empty((1, K), dtype=torch.int16, device="cuda")
+        sa = torch.empty(64, dtype=torch.float32, device="cuda")
+        y = torch.empty((1, N), dtype=torch.float16, device="cuda")
+        ws = workspace(torch, B, B.OP_GEMV, 1, K, N, 2, group)
+
+        def one_pass(with_quant):
+            for pk in packed:
+                if with_quant:
+                    B.tman_quantize_rows(x, 1, K, 32767, a, sa)
+                B.tman_mpgemv_ternary(pk, a, sa, 0.02, y, None, 1, K, N, group, ws)
+
+        res = {"leg": "ternary", "M": 1, "K": K, "N": N, "copies": ncopy, "plane_bytes": nbytes}
+        for with_quant in (False, True):
+            one_pass(True)
+            torch.cuda.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr):
+                for _ in range(4):
+                    one_pass(with_quant)
+            gr.replay()
+            torch.cuda.synchronize()
+            us = event_us(torch, gr.replay, reps)[0] / (4 * ncopy)
+            key = "us_with_quantize" if with_quant else "us"
+            res[key] = round(us, 2)
+            if not with_quant:
+                res["weight_stream_GBs"] = round(nbytes / us / 1e3, 1)
+        assert B.tman_read_status(ws) == 0
+        out.append(res)
+        del packed
+        torch.cuda.empty_cache()
+    return out
+
+
+def ternary(args, rest=()):
+    import torch
+    from paper_2511_11248_b200 import binding as B, helpers as H
+    for r in ternary_results(torch, B, H):
         print(json.dumps(r), flush=True)
 
 

@@ -137,6 +137,32 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed /*host*/, c
                                 const void *x_f16, void *const *y_f16 /*host*/, int M, int K, const int *N /*host*/,
                                 int bits, int group, void *workspace, size_t ws_bytes, tman_stream_t stream);
 
+/* ---- integer path: per-tensor ternary weights with 16-bit integer activations -------------------
+ * (paper Sec. 6.1 "Models and Quantization": BitNet's ternary weights, quantized per tensor, are treated
+ * as 2-bit, W_INT2 A_INT16; Sec. 4.3: integer aggregation inside the quantization block -- here the whole
+ * tensor -- and floating point after it.)
+ *
+ * Weights: codes q = t + 1 in {0, 1, 2} for t in {-1, 0, +1}, packed by tman_pack_weights with bits = 2
+ * (any legal group; the buffer's scales and zero-points are not read: zero-point 1 and the one scale
+ * w_scale are implied). */
+
+/* Per-row symmetric quantization of activations: row_scale[m] = max_k |x[m][k]| / qmax (1 for a row of
+ * zeros), a[m][k] = round(x[m][k] / row_scale[m]) clamped to +-qmax; division and rounding (to nearest
+ * even) in single precision.  qmax = 32767 (decode) or 127.  a_i16: int16 [M][K]; row_scale: fp32 [M]. */
+tman_status tman_quantize_rows(const void *x_f16, int M, int K, int qmax, int16_t *a_i16, float *row_scale,
+                               tman_stream_t stream);
+
+/* Decode of one row (M must be 1; K <= 16384): the bit-serial table lookup of tman_mpgemv on integers.
+ * Tables hold exact integer sums of activations, lookups are shift-accumulated, the activation sum is
+ * subtracted once (zero-point 1), K-slices are added as 32-bit integers;
+ *   y[n] = fp16( row_scale[0] * w_scale * sum_k a[k] * (q[k][n] - 1) ).
+ * acc_i32 (device, int32 [N], 16-byte aligned, may be NULL) receives the exact integer sums.
+ * Workspace and status word as for tman_mpgemv with M = 1. */
+tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const int16_t *a_i16,
+                                const float *row_scale, float w_scale, void *y_f16, int32_t *acc_i32,
+                                int M, int K, int N, int group,
+                                void *workspace, size_t ws_bytes, tman_stream_t stream);
+
 /* Prefill (paper Sec. 4.1 two-level LUT dequantization, Fig. 7; Sec. 4.2 three-stage pipeline,
  * Fig. 9): packed tiles are staged in shared memory, rebuilt into fp16 tiles through the
  * repack step and the per-(block, column) conversion table, and multiplied on the tensor

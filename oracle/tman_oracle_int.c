@@ -13,12 +13,12 @@
  *   weights      w[k][n] = s_w * t[k][n],  t in {-1, 0, +1},  stored as the 2-bit code q = t + 1
  *                (one scale s_w for the whole tensor; zero-point 1)
  *   activations  a[m][k] = round(x[m][k] / s_a[m]),  s_a[m] = max_k |x[m][k]| / QMAX
- *                (QMAX = 32767 for 16-bit decode, 127 for 8-bit prefill; x/s_a rounded to nearest,
- *                 ties to even; a row of zeros has s_a = 1 and a = 0)
+ *                (QMAX = 32767 for 16-bit decode, 127 for 8-bit prefill; both divisions in single
+ *                 precision, x/s_a rounded to nearest, ties to even; a row of zeros has s_a = 1, a = 0)
  *   result       y[m][n] = s_a[m] * s_w * sum_k a[m][k] * t[k][n]      (the sum is an exact integer)
  *
  * Readings taken where the paper is silent: the activation scale is per token (row) and symmetric;
- * rounding is to nearest even; the table entries of the bit-serial form are exact integer sums of four
+ * the scale and the quotient are single-precision values and rounding is to nearest even; the table entries of the bit-serial form are exact integer sums of four
  * activations; with one block per tensor the "inside the block" aggregation is the whole integer sum.
  *
  * Pins (see tests): the bit-serial table form equals the definition bit for bit; brute force on tiny
@@ -41,21 +41,26 @@ static double h2d(uint16_t h)
 }
 
 /* Per-token symmetric quantization of the activations (Sec. 6.1: A_INT16; INT8 for the matrix unit).
- * x: fp16 bits [M][K]; a: int32 [M][K] (values within +-qmax); s_a: fp64 [M]. */
+ * The scale and the quotient are computed in single precision (IEEE division, correctly rounded) and the
+ * quotient is rounded to the nearest integer, ties to even: floating point decides an integer here, so
+ * the precision is part of the definition, and single precision is what an accelerator kernel uses.
+ * x: fp16 bits [M][K]; a: int32 [M][K] (values within +-qmax); s_a: fp64 [M] (holding the fp32 value). */
 void oracle_quantize_rows(const uint16_t *x, int M, int K, int qmax, int32_t *a, double *s_a)
 {
     int m, k;
     for (m = 0; m < M; ++m) {
-        double amax = 0.0;
+        float amax = 0.0f, scale;
         for (k = 0; k < K; ++k) {
-            double v = fabs(h2d(x[(size_t)m * K + k]));
+            float v = fabsf((float)h2d(x[(size_t)m * K + k]));       /* fp16 -> fp32 is exact */
             if (v > amax) amax = v;
         }
-        s_a[m] = amax > 0.0 ? amax / (double)qmax : 1.0;
+        scale = amax > 0.0f ? amax / (float)qmax : 1.0f;
+        s_a[m] = (double)scale;
         for (k = 0; k < K; ++k) {
-            double r = nearbyint(h2d(x[(size_t)m * K + k]) / s_a[m]);     /* default mode: ties to even */
-            if (r > qmax) r = qmax;
-            if (r < -qmax) r = -qmax;
+            volatile float quot = (float)h2d(x[(size_t)m * K + k]) / scale;   /* one rounding, to fp32 */
+            float r = nearbyintf(quot);                                        /* default mode: ties to even */
+            if (r > (float)qmax) r = (float)qmax;
+            if (r < -(float)qmax) r = -(float)qmax;
             a[(size_t)m * K + k] = (int32_t)r;
         }
     }

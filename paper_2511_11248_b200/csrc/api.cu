@@ -149,6 +149,30 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed, const size
                                  reinterpret_cast<cudaStream_t>(stream));
 }
 
+tman_status tman_quantize_rows(const void *x_f16, int M, int K, int qmax, int16_t *a_i16, float *row_scale,
+                               tman_stream_t stream)
+{
+    if (!x_f16 || !a_i16 || !row_scale) return TMAN_ERR_NULL;
+    if (M < 1 || K < 1 || (qmax != 32767 && qmax != 127)) return TMAN_ERR_SHAPE;
+    if (!matrices_aligned(x_f16, a_i16)) return TMAN_ERR_SHAPE;
+    return launch_quantize_rows(x_f16, M, K, qmax, a_i16, row_scale, reinterpret_cast<cudaStream_t>(stream));
+}
+
+tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const int16_t *a_i16, const float *row_scale,
+                                float w_scale, void *y_f16, int32_t *acc_i32, int M, int K, int N, int group,
+                                void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    tman_status st = check_matmul(packed, packed_bytes, a_i16, y_f16, M, K, N, 2, group, workspace);
+    if (st != TMAN_OK) return st;
+    if (!row_scale) return TMAN_ERR_NULL;
+    if (M != 1) return TMAN_ERR_UNSUPPORTED;
+    if (K > 16384) return TMAN_ERR_UNSUPPORTED;            // 3 * K * 32767 must stay below the "no sum pending" pattern
+    if (acc_i32 && !aligned_to(acc_i32, 16)) return TMAN_ERR_SHAPE;
+    if (ws_bytes < mpgemv_workspace_bytes(1, K, N, 2)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_mpgemv_ternary(packed, a_i16, row_scale, w_scale, y_f16, acc_i32, K, N, group, workspace, ws_bytes,
+                                 reinterpret_cast<cudaStream_t>(stream));
+}
+
 tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream)

@@ -62,6 +62,12 @@ struct GemvParams {
     int col0[kGemvMaxGroup];                 // first concatenated column of each matrix
     int count;                               // matrices in this launch
     const __half   *x;          // first row of this launch
+    // integer path (per-tensor ternary weights, 16-bit integer activations): quantized activations,
+    // their per-row scales, the tensor's weight scale, optional exact integer sums [M][N]
+    const int16_t  *xi;
+    const float    *row_scale;
+    float           w_scale;
+    int32_t        *acc_out;
     float          *partials;
     uint32_t       *status;
     int M;                      // rows in this launch (<= MT)
@@ -76,8 +82,14 @@ struct GemvParams {
 // Transposing reduction over the lanes selected by MASK, 2*MASK, ..., below END: every stage
 // halves the number of values a lane keeps (or, once one is left, plainly adds).  `base` is the
 // logical index of vals[0].
-template <int N_, int MASK, int END>
+// INTS: the values are 32-bit integers kept in float registers (bit patterns) and are added as integers.
+template <int N_, int MASK, int END, bool INTS = false>
 struct LaneReduce {
+    static __device__ __forceinline__ float add(float a, float b)
+    {
+        if constexpr (INTS) return __int_as_float(__float_as_int(a) + __float_as_int(b));
+        else return a + b;
+    }
     static __device__ __forceinline__ void run(float *vals, int v, int &base)
     {
         if constexpr (MASK < END) {
@@ -88,13 +100,13 @@ struct LaneReduce {
                 for (int j = 0; j < H; ++j) {
                     const float keep = up ? vals[j + H] : vals[j];
                     const float send = up ? vals[j] : vals[j + H];
-                    vals[j] = keep + __shfl_xor_sync(0xffffffffu, send, MASK);
+                    vals[j] = add(keep, __shfl_xor_sync(0xffffffffu, send, MASK));
                 }
                 base += up ? H : 0;
-                LaneReduce<H, MASK * 2, END>::run(vals, v, base);
+                LaneReduce<H, MASK * 2, END, INTS>::run(vals, v, base);
             } else {
-                vals[0] += __shfl_xor_sync(0xffffffffu, vals[0], MASK);
-                LaneReduce<1, MASK * 2, END>::run(vals, v, base);
+                vals[0] = add(vals[0], __shfl_xor_sync(0xffffffffu, vals[0], MASK));
+                LaneReduce<1, MASK * 2, END, INTS>::run(vals, v, base);
             }
         }
     }
@@ -208,13 +220,19 @@ struct UnitRegs {
 // K-slice is first scaled by a power of two that brings its largest magnitude into [1, 2) (undone in
 // fp32 at the end), so that entries use fp16's range whatever the activations' size; the bits * 4
 // lookups of one plane word are accumulated in fp16 (low plane first), everything after that in fp32.
+// INT (one row, HALF): per-tensor ternary weights (2-bit codes, zero-point 1, one scale) with 16-bit integer
+// activations (paper Sec. 6.1: BitNet as W_INT2 A_INT16).  Tables hold exact integer sums (as fp32: a sum of
+// eight 16-bit values is below 2^24), a word's lookups and the pair sum stay exact in fp32, and from there
+// on the sums are 32-bit integers: the slice's lanes, the K-slices and the result are added as integers;
+// only the final product with the row's and the tensor's scale is floating point (Sec. 4.3).
 // ROLL: one set of unit registers; every strip's registers are refilled with the next unit's strip as
 // soon as its lookups are done (larger units, fewer per-unit fixed costs, same bytes in flight).
-template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL, int HR>
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL, int HR, int INT>
 __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     static_assert(!HALF || MT == 1, "half slices are for single-row tables");
+    static_assert(!INT || (HALF && !HR && !GROUPED && BITS == 2), "the integer path is built for one row of ternary weights");
     static_assert(!HR || !HALF, "fp16 row pairs use whole-warp or sub-warp slices");
     constexpr int R = HR ? 2 * MT : MT;    // activation rows of this launch
     constexpr int W = HALF ? 16 : 32 / MT; // plane words (lanes) per K-slice
@@ -285,8 +303,13 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
             r.w[s][i] = __ldcs(reinterpret_cast<const uint4 *>(q));
             q += row_bytes;
         }
-        r.sc[s] = __ldg(a.psc + (size_t)nb * (uint32_t)nblk);
-        r.z[s] = __ldg(a.pz + (size_t)nb * (uint32_t)nblk);
+        if constexpr (INT) {
+            r.sc[s] = make_uint2(0x3C003C00u, 0x3C003C00u);      // scale 1.0 four times (fp16), zero-point 1 four times
+            r.z[s] = 0x1111u;
+        } else {
+            r.sc[s] = __ldg(a.psc + (size_t)nb * (uint32_t)nblk);
+            r.z[s] = __ldg(a.pz + (size_t)nb * (uint32_t)nblk);
+        }
     };
     auto load_unit = [&](UnitRegs<BITS, S> &r, int wu) {
         const UnitAddr a = unit_addr(r, wu);
@@ -310,20 +333,35 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         const int slot = tid & 63, chunk = tid >> 6;
         const int gv = slot & 15, gc = slot >> 4;
         // index bit q of byte gc is word bit 8*gc + q, i.e. the weight 8*(q & 3) + 2*gc + (q >> 2)
-        __half2 raw[4];
-#pragma unroll
-        for (int ph = 0; ph < 4; ++ph) {
-            raw[ph] = __floats2half2_rn(0.f, 0.f);
-            if (gv < nwords)
-                raw[ph] = __ldg(reinterpret_cast<const __half2 *>(p.x + (size_t)(word0 + gv) * 32 + 8 * ph + 2 * gc));
-        }
-        if constexpr (!ROLL) load_unit(regs[1], wu0 + wstride);
         float xv[8];
+        if constexpr (INT) {
+            short2 raw[4];
 #pragma unroll
-        for (int ph = 0; ph < 4; ++ph) {
-            const float2 f = __half22float2(raw[ph]);
-            xv[ph] = f.x;
-            xv[ph + 4] = f.y;
+            for (int ph = 0; ph < 4; ++ph) {
+                raw[ph] = make_short2(0, 0);
+                if (gv < nwords)
+                    raw[ph] = __ldg(reinterpret_cast<const short2 *>(p.xi + (size_t)(word0 + gv) * 32 + 8 * ph + 2 * gc));
+            }
+#pragma unroll
+            for (int ph = 0; ph < 4; ++ph) {
+                xv[ph] = (float)raw[ph].x;
+                xv[ph + 4] = (float)raw[ph].y;
+            }
+        } else {
+            __half2 raw[4];
+#pragma unroll
+            for (int ph = 0; ph < 4; ++ph) {
+                raw[ph] = __floats2half2_rn(0.f, 0.f);
+                if (gv < nwords)
+                    raw[ph] = __ldg(reinterpret_cast<const __half2 *>(p.x + (size_t)(word0 + gv) * 32 + 8 * ph + 2 * gc));
+            }
+            if constexpr (!ROLL) load_unit(regs[1], wu0 + wstride);
+#pragma unroll
+            for (int ph = 0; ph < 4; ++ph) {
+                const float2 f = __half22float2(raw[ph]);
+                xv[ph] = f.x;
+                xv[ph + 4] = f.y;
+            }
         }
         float lo[16];
         lut16(xv[0], xv[1], xv[2], xv[3], lo);
@@ -594,8 +632,12 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 }
             }
         }
-        // the other lanes of the K-slice
-        LaneReduce<V1, PRE ? 2 : 1, W>::run(vals, v, base);
+        // the other lanes of the K-slice (integer path: exact integers so far, added as integers from here on)
+        if constexpr (INT) {
+#pragma unroll
+            for (int e = 0; e < V1; ++e) vals[e] = __int_as_float(__float2int_rn(vals[e]));
+        }
+        LaneReduce<V1, PRE ? 2 : 1, W, INT != 0>::run(vals, v, base);
         const bool writer = (V >= W) ? true : (v < V);
         if (writer && wu < p.units) {
             const int g = GROUPED ? g_u : 0;
@@ -606,8 +648,16 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 if (n < lim && m < p.M) {
                     float out = vals[e];
                     if constexpr (HR) out *= reinterpret_cast<const float *>(smem + kGemvTableBytes)[m];   // undo the row's scale
-                    if (p.nkappa == 1) p.y[g][(size_t)m * p.Ng[g] + (n - (GROUPED ? p.col0[g] : 0))] = __float2half_rn(out);
-                    else p.partials[((size_t)kappa * R + m) * p.N + n] = out;
+                    if (p.nkappa == 1) {
+                        if constexpr (INT) {
+                            const int acc = __float_as_int(out);
+                            if (p.acc_out) p.acc_out[(size_t)m * p.N + n] = acc;
+                            out = (float)acc * (__ldg(p.row_scale + m) * p.w_scale);
+                        }
+                        p.y[g][(size_t)m * p.Ng[g] + (n - (GROUPED ? p.col0[g] : 0))] = __float2half_rn(out);
+                    } else {
+                        p.partials[((size_t)kappa * R + m) * p.N + n] = out;     // integer path: the integer's bit pattern
+                    }
                 }
             }
         }
@@ -640,30 +690,40 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
         while (SP < 8 && 2 * SP <= p.nkappa && items * 2 * SP <= kGemvThreads) SP *= 2;
         const int part = tid & (SP - 1);
         const float sv = __uint_as_float(kGemvSentinel);
+        using RED = LaneReduce<1, 1, 1, INT != 0>;          // its add(): floats, or integers kept in float registers
         bool gave_up = false;
         for (int item0 = 0; item0 < items; item0 += kGemvThreads / SP) {
             const int item = item0 + tid / SP;
             const bool alive = item < items;
             const int m = alive ? item / ngrp : 0, n = col_lo + 4 * (alive ? item % ngrp : 0);
             float4 *src = reinterpret_cast<float4 *>(p.partials + (size_t)m * p.N + n);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);      // also the bit pattern of integer zero
             for (int kp = part; alive && kp < p.nkappa; kp += 4 * SP) {
                 float4 t[4];
                 if (!wait_for_sums(src, stride4, kp, SP, p.nkappa, kGemvPollLimit, t)) { gave_up = true; break; }
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     if (kp + q * SP < p.nkappa) {
-                        acc.x += t[q].x; acc.y += t[q].y; acc.z += t[q].z; acc.w += t[q].w;
+                        acc.x = RED::add(acc.x, t[q].x); acc.y = RED::add(acc.y, t[q].y);
+                        acc.z = RED::add(acc.z, t[q].z); acc.w = RED::add(acc.w, t[q].w);
                         src[(size_t)(kp + q * SP) * stride4] = make_float4(sv, sv, sv, sv);
                     }
             }
             for (int mask = 1; mask < SP; mask <<= 1) {
-                acc.x += __shfl_xor_sync(0xffffffffu, acc.x, mask);
-                acc.y += __shfl_xor_sync(0xffffffffu, acc.y, mask);
-                acc.z += __shfl_xor_sync(0xffffffffu, acc.z, mask);
-                acc.w += __shfl_xor_sync(0xffffffffu, acc.w, mask);
+                acc.x = RED::add(acc.x, __shfl_xor_sync(0xffffffffu, acc.x, mask));
+                acc.y = RED::add(acc.y, __shfl_xor_sync(0xffffffffu, acc.y, mask));
+                acc.z = RED::add(acc.z, __shfl_xor_sync(0xffffffffu, acc.z, mask));
+                acc.w = RED::add(acc.w, __shfl_xor_sync(0xffffffffu, acc.w, mask));
             }
             gave_up = __any_sync(0xffffffffu, gave_up);
+            if constexpr (INT) {
+                if (alive && part == 0 && !gave_up) {
+                    const int4 ia = make_int4(__float_as_int(acc.x), __float_as_int(acc.y), __float_as_int(acc.z), __float_as_int(acc.w));
+                    if (p.acc_out) *reinterpret_cast<int4 *>(p.acc_out + (size_t)m * p.N + n) = ia;
+                    const float sc = __ldg(p.row_scale + m) * p.w_scale;
+                    acc = make_float4((float)ia.x * sc, (float)ia.y * sc, (float)ia.z * sc, (float)ia.w * sc);
+                }
+            }
             if (alive && part == 0 && !gave_up) {
                 const __half2 h01 = __floats2half2_rn(acc.x, acc.y), h23 = __floats2half2_rn(acc.z, acc.w);
                 uint2 o;
@@ -681,7 +741,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
     }
 }
 
-template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL, int HR>
+template <int BITS, int MT, int S, int PRE, int HALF, int GROUPED, int ROLL, int HR, int INT = 0>
 static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
 {
     constexpr int W = HALF ? 16 : 32 / MT;
@@ -706,7 +766,7 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
         cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev) != cudaSuccess)
         return TMAN_ERR_CUDA;
     if ((uint32_t)reserved != kGemvSmemBase) return TMAN_ERR_UNSUPPORTED;
-    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED, ROLL, HR>;
+    auto kern = mpgemv_kernel<BITS, MT, S, PRE, HALF, GROUPED, ROLL, HR, INT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
         return TMAN_ERR_CUDA;
     // the grid has at most one CTA per SM; the occupancy query says whether an SM can hold one at all
@@ -914,6 +974,7 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
     }
     p.status = reinterpret_cast<uint32_t *>(w8);
     p.partials = reinterpret_cast<float *>(w8 + kWsStatusBytes);
+    p.xi = nullptr; p.row_scale = nullptr; p.w_scale = 0.f; p.acc_out = nullptr;
     p.K = K; p.bits = bits; p.group = group;
     p.M = 0; p.nkappa = 0; p.P = 0; p.units = 0;
     p.group_shift = (group == 32) ? 5 : (group == 64) ? 6 : 7;
@@ -933,6 +994,101 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
         m0 += rows;
     }
     return TMAN_OK;
+}
+
+// ---- integer path: per-tensor ternary weights, 16-bit integer activations ---------------------------
+// Per-row symmetric quantization of the activations (paper Sec. 6.1, A_INT16; 8 bits for the matrix unit):
+// s_a = max|x| / qmax and a = round(x / s_a), both in single precision with correctly rounded division and
+// rounding to nearest even, so that the integers are the same on any IEEE machine.  One CTA per row.
+__global__ void __launch_bounds__(1024) quantize_rows_kernel(const __half *__restrict__ x, int K, int qmax,
+                                                             int16_t *__restrict__ a, float *__restrict__ s_a)
+{
+    __shared__ float red[32];
+    const __half *row = x + (size_t)blockIdx.x * K;
+    int16_t *out = a + (size_t)blockIdx.x * K;
+    // eight values per thread and step when the row allows 16-byte accesses (K % 8 == 0, checked by the host)
+    const bool vec = (K & 7) == 0;
+    const int nvec = vec ? K >> 3 : 0;
+    float amax = 0.f;
+    for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4 *>(row) + i);
+        const __half2 *h = reinterpret_cast<const __half2 *>(&q);
+        __half2 m = __hmax2(__hmax2(__habs2(h[0]), __habs2(h[1])), __hmax2(__habs2(h[2]), __habs2(h[3])));
+        amax = fmaxf(amax, fmaxf(__low2float(m), __high2float(m)));
+    }
+    for (int k = 8 * nvec + threadIdx.x; k < K; k += blockDim.x) amax = fmaxf(amax, fabsf(__half2float(row[k])));
+    for (int mask = 16; mask > 0; mask >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, mask));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+        for (int mask = 16; mask > 0; mask >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, mask));
+        if (threadIdx.x == 0) red[0] = v;
+    }
+    __syncthreads();
+    amax = red[0];
+    const float scale = amax > 0.f ? __fdiv_rn(amax, (float)qmax) : 1.f;
+    if (threadIdx.x == 0) s_a[blockIdx.x] = scale;
+    auto quant = [&](__half v) {
+        const int r = __float2int_rn(__fdiv_rn(__half2float(v), scale));
+        return (int)max(-qmax, min(qmax, r));
+    };
+    for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4 *>(row) + i);        // second read: from L1/L2
+        const __half *h = reinterpret_cast<const __half *>(&q);
+        uint4 o;
+        o.x = (uint32_t)(quant(h[0]) & 0xFFFF) | ((uint32_t)quant(h[1]) << 16);
+        o.y = (uint32_t)(quant(h[2]) & 0xFFFF) | ((uint32_t)quant(h[3]) << 16);
+        o.z = (uint32_t)(quant(h[4]) & 0xFFFF) | ((uint32_t)quant(h[5]) << 16);
+        o.w = (uint32_t)(quant(h[6]) & 0xFFFF) | ((uint32_t)quant(h[7]) << 16);
+        reinterpret_cast<uint4 *>(out)[i] = o;
+    }
+    for (int k = 8 * nvec + threadIdx.x; k < K; k += blockDim.x) out[k] = (int16_t)quant(row[k]);
+}
+
+tman_status launch_quantize_rows(const void *x, int M, int K, int qmax, int16_t *a, float *s_a, cudaStream_t s)
+{
+    const int threads = K >= 8192 ? 1024 : (K >= 2048 ? 512 : 256);
+    quantize_rows_kernel<<<(unsigned)M, threads, 0, s>>>(static_cast<const __half *>(x), K, qmax, a, s_a);
+    return launch_status();
+}
+
+// One row of 16-bit integer activations times ternary weights packed as 2-bit codes (zero-point 1; the
+// packed buffer's scales and zero-points are not read).  y = fp16(s_a * s_w * sum), acc_out (may be NULL)
+// receives the exact integer sums.
+tman_status launch_mpgemv_ternary(const void *packed, const int16_t *a, const float *s_a, float s_w, void *y,
+                                  int32_t *acc_out, int K, int N, int group, void *ws, size_t, cudaStream_t s)
+{
+    const int sms = sm_count();
+    if (sms <= 0) return TMAN_ERR_CUDA;
+    if (!variant_feasible(kGemvVariants[0], K, N, sms, (size_t)-1)) return TMAN_ERR_UNSUPPORTED;
+    uint8_t *w8 = static_cast<uint8_t *>(ws);
+    GemvParams p = {};
+    p.count = 1;
+    Layout L = make_layout(K, N, 2, group);
+    const uint8_t *pk = static_cast<const uint8_t *>(packed);
+    for (int g = 0; g < kGemvMaxGroup; ++g) {
+        p.packed[g] = pk;
+        p.planes[g] = reinterpret_cast<const uint4 *>(pk + L.planes_off);
+        p.scales[g] = reinterpret_cast<const uint2 *>(pk + L.scales_off);
+        p.zeros[g] = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
+        p.Ng[g] = g == 0 ? N : 0;
+        p.col0[g] = g == 0 ? 0 : N;
+        p.y[g] = static_cast<__half *>(y);
+    }
+    p.N = N;
+    p.x = nullptr;
+    p.xi = a;
+    p.row_scale = s_a;
+    p.w_scale = s_w;
+    p.acc_out = acc_out;
+    p.status = reinterpret_cast<uint32_t *>(w8);
+    p.partials = reinterpret_cast<float *>(w8 + kWsStatusBytes);
+    p.K = K; p.bits = 2; p.group = group; p.M = 1;
+    p.group_shift = (group == 32) ? 5 : (group == 64) ? 6 : 7;
+    p.nblk = K / group;
+    if (group >= 64) return launch_one<2, 1, 4, 1, 1, 0, 1, 0, 1>(p, sms, s);
+    return launch_one<2, 1, 4, 0, 1, 0, 1, 0, 1>(p, sms, s);
 }
 
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,

@@ -20,10 +20,13 @@ def test_row_quantization_by_hand():
     # Sec. 6.1 (A_INT16): one row by hand: amax = 2 -> s_a = 2 / 32767; ties go to the even integer
     x = np.array([[2.0, -1.0, 0.5, 0.0]], dtype=np.float16)
     a, s = oi.quantize_rows(x, 32767)
-    assert s[0] == 2.0 / 32767
+    assert s[0] == float(np.float32(2.0) / np.float32(32767))            # the scale is a single-precision value
     assert a.tolist() == [[32767, -16384, 8192, 0]]      # 16383.5 -> 16384 (even), 8191.75 -> 8192
     a8, s8 = oi.quantize_rows(x, 127)
-    assert s8[0] == 2.0 / 127 and a8.tolist() == [[127, -64, 32, 0]]   # 63.5 -> 64 (even), 31.75 -> 32
+    assert s8[0] == float(np.float32(2.0) / np.float32(127)) and a8.tolist() == [[127, -64, 32, 0]]   # 63.5 -> 64, 31.75 -> 32
+    # an exact tie decided in single precision: amax = 127 -> s_a = 1, 2.5 -> 2 and 3.5 -> 4 (to even)
+    a8, s8 = oi.quantize_rows(np.array([[127.0, 2.5, 3.5, -2.5]], dtype=np.float16), 127)
+    assert s8[0] == 1.0 and a8.tolist() == [[127, 2, 4, -2]]
     # an all-zero row keeps scale 1 and quantizes to zeros
     a0, s0 = oi.quantize_rows(np.zeros((1, 8), dtype=np.float16), 32767)
     assert s0[0] == 1.0 and not a0.any()
@@ -35,9 +38,11 @@ def test_row_quantization_properties(qmax):
     a, s = oi.quantize_rows(x, qmax)
     xf = x.astype(np.float64)
     assert np.all(np.abs(a) <= qmax) and np.all(np.abs(a).max(axis=1) == qmax)
-    assert np.allclose(s, np.abs(xf).max(axis=1) / qmax, rtol=0, atol=0)
-    assert np.all(np.abs(xf - a * s[:, None]) <= s[:, None] / 2 * (1 + 1e-12))
-    assert np.array_equal(a, np.rint(xf / s[:, None]).astype(np.int32))       # numpy rounds ties to even too
+    s32 = (np.abs(x.astype(np.float32)).max(axis=1) / np.float32(qmax)).astype(np.float32)
+    assert np.array_equal(s, s32.astype(np.float64))                           # single-precision scale
+    # half a step, plus the single-precision quotient's own rounding (at most 2^-9 of a step near qmax)
+    assert np.all(np.abs(xf - a * s[:, None]) <= s[:, None] * (0.5 + 2.0 ** -8))
+    assert np.array_equal(a, np.rint(x.astype(np.float32) / s32[:, None]).astype(np.int32))   # fp32 quotient, ties to even
 
 
 def test_definition_against_brute_force_and_numpy():
@@ -101,7 +106,7 @@ def test_result_within_the_quantization_error_bound(qmax, fn):
     exact = s_w * (x.astype(np.float64) @ t.astype(np.float64))
     _, s_a = oi.quantize_rows(x, qmax)
     bound = s_w * (s_a[:, None] / 2) * np.abs(t).sum(axis=0, dtype=np.float64)[None, :]
-    assert np.all(np.abs(y - exact) <= bound * (1 + 1e-9) + 1e-12)
+    assert np.all(np.abs(y - exact) <= bound * (1 + 2.0 ** -7) + 1e-12)
     # and the 16-bit path is far inside the fp path's tolerance, the 8-bit path is not as close
     rel = np.max(np.abs(y - exact)) / np.max(np.abs(exact))
     assert rel < (1e-4 if qmax == 32767 else 2e-2)
