@@ -345,8 +345,27 @@ def ternary_results(torch, B, H, reps=7):
             if not with_quant:
                 res["weight_stream_GBs"] = round(nbytes / us / 1e3, 1)
         assert B.tman_read_status(ws) == 0
+        # the prefill side's dequantization step alone: packed planes -> INT8 [N][K]
+        w8 = [torch.empty((N, K), dtype=torch.int8, device="cuda") for _ in range(min(ncopy, 16))]
+        wsd = workspace(torch, B, B.OP_AUX, 1, K, N, 2, group)
+
+        def dq():
+            for i, pk in enumerate(packed):
+                B.tman_dequant_ternary_int8(pk, K, N, group, w8[i % len(w8)], wsd)
+
+        dq()
+        torch.cuda.synchronize()
+        gd = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gd):
+            dq()
+        gd.replay()
+        torch.cuda.synchronize()
+        us = event_us(torch, gd.replay, reps)[0] / ncopy
+        assert B.tman_read_status(wsd) == 0
+        res["dequant_int8_us"] = round(us, 2)
+        res["dequant_int8_GBs"] = round((nbytes + K * N) / us / 1e3, 1)      # planes read + INT8 written
         out.append(res)
-        del packed
+        del packed, w8
         torch.cuda.empty_cache()
     return out
 

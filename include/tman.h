@@ -163,6 +163,15 @@ tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const i
                                 int M, int K, int N, int group,
                                 void *workspace, size_t ws_bytes, tman_stream_t stream);
 
+/* Prefill side of the integer path, the dequantization step alone (paper Sec. 6.2 "mpGEMM": per-tensor
+ * weights are dequantized to INT8 for the matrix unit; Sec. 4.1 / Fig. 7: by two table lookups, bit
+ * repacking and a conversion table, here with the INT8 values -1, 0, +1 as the table's entries).
+ * w8_nk: output, int8 [N][K] (channel-major, 16-byte aligned).  workspace: at least 256 bytes (status
+ * word: a header that does not match leaves the output untouched).  The INT8 matrix multiplication that
+ * would consume these tiles on the tensor cores is not part of the library. */
+tman_status tman_dequant_ternary_int8(const void *packed, size_t packed_bytes, int K, int N, int group,
+                                      int8_t *w8_nk, void *workspace, size_t ws_bytes, tman_stream_t stream);
+
 /* Prefill (paper Sec. 4.1 two-level LUT dequantization, Fig. 7; Sec. 4.2 three-stage pipeline,
  * Fig. 9): packed tiles are staged in shared memory, rebuilt into fp16 tiles through the
  * repack step and the per-(block, column) conversion table, and multiplied on the tensor

@@ -23,7 +23,7 @@ EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
     "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
-    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for", "tman_debug_gemv_plan", "tman_debug_wait_timeout", "tman_debug_mpgemm_variant", "tman_quantize_rows", "tman_mpgemv_ternary",
+    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for", "tman_debug_gemv_plan", "tman_debug_wait_timeout", "tman_debug_mpgemm_variant", "tman_quantize_rows", "tman_mpgemv_ternary", "tman_dequant_ternary_int8",
 ]
 
 _lib = None
@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
         L.tman_debug_gemm_plan_for.argtypes = [i, i, i, i, i, i, i, C.POINTER(C.c_int)]
         L.tman_debug_gemv_plan.argtypes = [i, i, i, i, i, i, sz, C.POINTER(C.c_int)]
         L.tman_debug_wait_timeout.argtypes = [vp, sz, C.c_uint, vp]
+        L.tman_dequant_ternary_int8.argtypes = [vp, sz, i, i, i, vp, vp, sz, vp]
         L.tman_quantize_rows.argtypes = [vp, i, i, i, vp, vp, vp]
         L.tman_mpgemv_ternary.argtypes = [vp, sz, vp, vp, C.c_float, vp, vp, i, i, i, i, vp, sz, vp]
         L.tman_debug_mpgemm_variant.argtypes = [i, vp, sz, vp, vp, i, i, i, i, i, vp, vp, sz, vp]
@@ -191,6 +192,12 @@ def tman_debug_gemv_plan(M, K, N, bits, group, sms=148, ws_limit=0) -> dict:
     keys = ("rows", "variant_rows", "words", "slices", "ctas", "smem_bytes")
     return {"ws_kib": out[1], "cost_us": out[2] / 1000.0,
             "passes": [dict(zip(keys, out[4 + 6 * i: 10 + 6 * i])) for i in range(out[0])]}
+
+
+def tman_dequant_ternary_int8(packed, K, N, group, w8, ws, stream=None) -> None:
+    _check(lib().tman_dequant_ternary_int8(_ptr(packed), packed.numel() * packed.element_size(), K, N, group, _ptr(w8),
+                                           _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "tman_dequant_ternary_int8")
 
 
 def tman_quantize_rows(x, M, K, qmax, a, row_scale, stream=None) -> None:

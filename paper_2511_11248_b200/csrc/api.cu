@@ -173,6 +173,19 @@ tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const i
                                  reinterpret_cast<cudaStream_t>(stream));
 }
 
+tman_status tman_dequant_ternary_int8(const void *packed, size_t packed_bytes, int K, int N, int group, int8_t *w8_nk,
+                                      void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    if (!packed || !w8_nk || !workspace) return TMAN_ERR_NULL;
+    tman_status st = check_format(K, N, 2, group);
+    if (st != TMAN_OK) return st;
+    if (packed_bytes < make_layout(K, N, 2, group).total) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
+    if (!buffers_aligned(packed, workspace) || !aligned_to(w8_nk, 16)) return TMAN_ERR_SHAPE;
+    return launch_dequant_ternary_int8(packed, K, N, group, w8_nk, static_cast<uint32_t *>(workspace),
+                                       reinterpret_cast<cudaStream_t>(stream));
+}
+
 tman_status tman_mpgemm(const void *packed, size_t packed_bytes, const void *x_f16, void *y_f16,
                         int M, int K, int N, int bits, int group,
                         void *workspace, size_t ws_bytes, tman_stream_t stream)

@@ -111,6 +111,8 @@ tman_status launch_pack(const uint8_t *codes, const void *scales, const uint8_t 
 // dependent launch): note_packed_write records the stream, packed_write_pending asks and clears.
 void note_packed_write(cudaStream_t s);
 bool packed_write_pending(cudaStream_t s, bool clear);
+tman_status launch_dequant_ternary_int8(const void *packed, int K, int N, int group, int8_t *w8, uint32_t *status,
+                                        cudaStream_t s);
 tman_status launch_unpack(const void *packed, int K, int N, int bits, int group, uint8_t *codes,
                           void *scales, uint8_t *zeros, uint32_t *status, cudaStream_t s);
 tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int group, uint8_t *idx,

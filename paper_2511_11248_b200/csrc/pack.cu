@@ -197,6 +197,62 @@ __global__ void debug_indices_kernel(const uint8_t *__restrict__ packed, uint8_t
     }
 }
 
+// ---- per-tensor ternary weights -> INT8 by two table lookups (paper Sec. 4.1 / Fig. 7, Sec. 6.2) -----------
+// One thread takes the two plane words of 32 consecutive k of the four columns of a strip.  Level 1 (bit
+// repacking): the planes are interleaved into 2-bit codes, eight to a register in k order, one code per
+// nibble (the packed format's bit permutation makes a shift and a bit-select do it).  Level 2 (conversion
+// table): a four-entry byte table {-1, 0, +1, 0} held in one register, looked up four codes at a time with
+// a byte permute whose selector is the codes themselves.  Output: int8 [N][K], 32 bytes per thread and
+// column, consecutive threads on consecutive k.
+__global__ void dequant_ternary_int8_kernel(const uint8_t *__restrict__ packed, int8_t *__restrict__ w8,
+                                            uint32_t *status, int K, int N, int group)
+{
+    if (!header_matches(packed, K, N, 2, group)) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
+        return;
+    }
+    const Layout L = make_layout(K, N, 2, group);
+    const int words = K / 32;
+    const long tid = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (tid >= (long)(N / 4) * words) return;
+    const int nb = (int)(tid / words), v = (int)(tid % words);
+    const uint4 *planes = reinterpret_cast<const uint4 *>(packed + L.planes_off);
+    const uint4 w0 = __ldg(planes + ((size_t)nb * 2 + 0) * words + v);
+    const uint4 w1 = __ldg(planes + ((size_t)nb * 2 + 1) * words + v);
+    const uint32_t table = 0x000100FFu;              // byte c = value of code c: -1, 0, +1, (3 does not occur) 0
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t p0 = c == 0 ? w0.x : c == 1 ? w0.y : c == 2 ? w0.z : w0.w;
+        const uint32_t p1 = c == 0 ? w1.x : c == 1 ? w1.y : c == 2 ? w1.z : w1.w;
+        // word bit 4j + ph belongs to weight 8ph + j: a0 holds, in its even bit pairs... interleave planes bit by bit
+        const uint32_t a0 = (p0 & 0x55555555u) | ((p1 << 1) & 0xAAAAAAAAu);      // codes of the even word bits
+        const uint32_t a1 = ((p0 >> 1) & 0x55555555u) | (p1 & 0xAAAAAAAAu);      // codes of the odd word bits
+        uint32_t X[4];                               // X[ph]: nibble j = code of weight 8ph + j
+        X[0] = a0 & 0x33333333u;
+        X[2] = (a0 >> 2) & 0x33333333u;
+        X[1] = a1 & 0x33333333u;
+        X[3] = (a1 >> 2) & 0x33333333u;
+        uint32_t out[8];
+#pragma unroll
+        for (int ph = 0; ph < 4; ++ph) {
+            out[2 * ph] = __byte_perm(table, 0u, X[ph]);             // weights 8ph .. 8ph+3
+            out[2 * ph + 1] = __byte_perm(table, 0u, X[ph] >> 16);   // weights 8ph+4 .. 8ph+7
+        }
+        uint4 *dst = reinterpret_cast<uint4 *>(w8 + ((size_t)(4 * nb + c) * K + (size_t)32 * v));
+        dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+        dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+    }
+}
+
+tman_status launch_dequant_ternary_int8(const void *packed, int K, int N, int group, int8_t *w8, uint32_t *status,
+                                        cudaStream_t s)
+{
+    const long total = (long)(N / 4) * (K / 32);
+    dequant_ternary_int8_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(static_cast<const uint8_t *>(packed), w8,
+                                                                             status, K, N, group);
+    return launch_status();
+}
+
 tman_status launch_debug_indices(const void *packed, int K, int N, int bits, int group, uint8_t *idx,
                                  uint32_t *status, cudaStream_t s)
 {

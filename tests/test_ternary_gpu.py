@@ -103,3 +103,23 @@ def test_ternary_closed_forms_and_refusals():
     y.fill_(3.0)
     B.tman_mpgemv_ternary(junk, a, s, s_w, y, acc, 1, K, N, 64, ws)
     assert B.tman_read_status(ws) == 5 and bool((y == 3.0).all())
+
+
+@pytest.mark.parametrize("K,N,group", [(128, 8, 128), (2560, 2560, 128), (6912, 2560, 64), (1152, 264, 32)])
+def test_int8_dequantization_is_bit_exact(K, N, group):
+    # Sec. 6.2: per-tensor weights become INT8 through the two lookups; compared with the oracle's tables
+    _, t, q, _ = ternary_case(1, K, N, seed=K * 3 + N)
+    packed = pack_ternary(q, group)
+    ws = H.alloc_workspace(B.OP_AUX, 1, K, N, 2, group)
+    w8 = H.guarded_bytes(K * N, "w8").view(torch.int8).view(N, K)
+    w8.fill_(55)
+    B.tman_dequant_ternary_int8(packed, K, N, group, w8, ws)
+    assert B.tman_read_status(ws) == 0
+    H.check_guards()
+    want = oi.ternary_dequant_int8(q)                         # [K][N]
+    assert np.array_equal(w8.cpu().numpy().T, want)
+    # a buffer of another shape is refused and the output stays as it was
+    w8.fill_(55)
+    other = pack_ternary(np.ones((K, N + 8), dtype=np.uint8), group)
+    B.tman_dequant_ternary_int8(other, K, N, group, w8, ws)
+    assert B.tman_read_status(ws) == 5 and bool((w8 == 55).all())
