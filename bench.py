@@ -551,7 +551,7 @@ def main():
     ap.add_argument("--skip-gemm", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-sweeps", action="store_true", help="leave the config 1/3/5 digests out of the line")
-    ap.add_argument("--leg", default="headline", choices=["headline", "case", "config1", "config3", "config5", "ablation", "ternary", "microbench"],
+    ap.add_argument("--leg", default="headline", choices=["headline", "case", "config1", "config3", "config5", "ablation", "ternary", "stamps", "microbench"],
                     help="headline: the bench line (default); the others print their own JSON lines")
     args, rest = ap.parse_known_args()
     if args.leg != "headline":

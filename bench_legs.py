@@ -7,6 +7,7 @@
     python bench.py --leg ternary                  # integer decode: ternary weights, 16-bit integer activations, BitNet sizes
     python bench.py --leg ablation                 # prefill with ConvertDQ / LoadFull / sequential in place of the product path
     python bench.py --leg microbench               # lookup rates, load paths, cluster exchange
+    TMAN_LIBRARY=paper_2511_11248_b200/libtman_stamps.so python bench.py --leg stamps   # where the prefill roles wait
 
 Everything goes through the C ABI; one JSON line per result on stdout.  Weights and activations are
 seeded synthetic data drawn on the device (timing does not depend on the values; parity is the tests'
@@ -421,6 +422,38 @@ def ablation(args, rest=()):
     from paper_2511_11248_b200 import binding as B, helpers as H
     for r in ablation_results(torch, B, H):
         print(json.dumps(r), flush=True)
+
+
+# ---- role time stamps of the prefill kernel (needs TMAN_LIBRARY=.../libtman_stamps.so) -------------------
+
+def stamps(args, rest=()):
+    """Where each role of the prefill pipeline waits (paper Sec. 4.2, Fig. 9).  Run as
+    TMAN_LIBRARY=paper_2511_11248_b200/libtman_stamps.so python bench.py --leg stamps"""
+    import torch
+    from paper_2511_11248_b200 import binding as B, helpers as H
+    for M, K, N, bits in ((1024, 4096, 14336, 4), (1024, 4096, 4096, 4), (2048, 3584, 18944, 4), (128, 3584, 18944, 4),
+                          (1024, 4096, 14336, 2)):
+        group = 128
+        packed, x = device_problem(torch, B, H, M, K, N, bits, group, seed=3)
+        ws = workspace(torch, B, B.OP_GEMM, M, K, N, bits, group)
+        y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        for _ in range(3):
+            B.tman_mpgemm(packed, x, y, M, K, N, bits, group, ws)
+        torch.cuda.synchronize()
+        assert B.tman_read_status(ws) == 0
+        plan = B.tman_debug_gemm_plan(M, K, N, bits, group)
+        ctas = plan["workers"] * (2 if plan["pair"] else 1)
+        st = B.tman_debug_role_stamps(ws, ctas).astype(np.float64)
+        role = lambda w0, w1, col: float(np.median(st[:, w0:w1, col] / st[:, w0:w1, 2]))
+        lead = st[::2] if plan["pair"] else st                 # in a pair only the first CTA issues the MMAs
+        print(json.dumps({
+            "leg": "stamps", "M": M, "K": K, "N": N, "bits": bits, "group": group, "ctas": ctas, "pair": plan["pair"],
+            "role_clocks_median": float(np.median(st[:, 0, 2])),
+            "producer_waits_for_free_stage": round(role(0, 1, 0), 3),
+            "mma_waits_for_free_accumulators": round(float(np.median(lead[:, 1, 0] / lead[:, 1, 2])), 3),
+            "mma_waits_for_dequantized_stage": round(float(np.median(lead[:, 1, 1] / lead[:, 1, 2])), 3),
+            "dequant_waits_for_loaded_stage": round(role(2, 18, 0), 3),
+            "epilogue_waits_for_accumulators": round(role(18, 26, 0), 3)}), flush=True)
 
 
 # ---- digests for the headline line ------------------------------------------------------------------

@@ -243,6 +243,18 @@ tman_status tman_debug_mpgemm_variant(int variant, const void *packed, size_t pa
                                       void *y_f16, int M, int K, int N, int bits, int group, const void *wt_f16,
                                       void *workspace, size_t ws_bytes, tman_stream_t stream);
 
+/* Role time stamps of the last tman_mpgemm call on `workspace` (paper Sec. 4.2, Fig. 9: how long each
+ * of the three pipeline agents waits for the others).  Only a library built with -DTMAN_ROLE_STAMPS
+ * (python -m paper_2511_11248_b200.build --stamps -> libtman_stamps.so) records them: clock readings
+ * around every role's barrier waits, nothing else changes and the results are the same bits; the
+ * regular library returns TMAN_ERR_UNSUPPORTED.  out_host: ctas x 26 warps x 4 int64 (host): clocks
+ * in the warp's first kind of wait, in its second kind, in the whole role, and a tag.  Warp 0 (TMA
+ * producer) waits for a free stage; warp 1 (MMA issuer) for free accumulators / for a dequantized stage;
+ * warps 2-17 (dequantization) for a loaded stage; warps 18-25 (epilogue) for complete accumulators.
+ * Waits for the stream. */
+tman_status tman_debug_role_stamps(const void *workspace, size_t ws_bytes, int ctas, long long *out_host /*host*/,
+                                   tman_stream_t stream);
+
 /* How tman_mpgemm would cut a call's work on the current device (host-side decision, nothing is
  * launched; no counterpart in the paper).  out8 (host) receives: 1 if pairs of CTAs work on a tile
  * else 0; 128-token row blocks per CTA; row tiles; column tiles; 1 if every tile is dealt whole

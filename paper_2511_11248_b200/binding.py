@@ -10,7 +10,8 @@ import ctypes as C
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libtman.so")
+# TMAN_LIBRARY selects another build of the same library (e.g. libtman_stamps.so, the build with role time stamps)
+LIB_PATH = os.environ.get("TMAN_LIBRARY") or os.path.join(HERE, "libtman.so")
 
 TMAN_OK = 0
 STATUS_NAMES = {
@@ -23,7 +24,7 @@ EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
     "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
-    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for", "tman_debug_gemv_plan", "tman_debug_wait_timeout", "tman_debug_mpgemm_variant", "tman_quantize_rows", "tman_mpgemv_ternary", "tman_dequant_ternary_int8",
+    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for", "tman_debug_gemv_plan", "tman_debug_wait_timeout", "tman_debug_mpgemm_variant", "tman_quantize_rows", "tman_mpgemv_ternary", "tman_dequant_ternary_int8", "tman_debug_role_stamps",
 ]
 
 _lib = None
@@ -66,6 +67,7 @@ def lib() -> C.CDLL:
         L.tman_debug_gemm_plan_for.argtypes = [i, i, i, i, i, i, i, C.POINTER(C.c_int)]
         L.tman_debug_gemv_plan.argtypes = [i, i, i, i, i, i, sz, C.POINTER(C.c_int)]
         L.tman_debug_wait_timeout.argtypes = [vp, sz, C.c_uint, vp]
+        L.tman_debug_role_stamps.argtypes = [vp, sz, i, vp, vp]
         L.tman_dequant_ternary_int8.argtypes = [vp, sz, i, i, i, vp, vp, sz, vp]
         L.tman_quantize_rows.argtypes = [vp, i, i, i, vp, vp, vp]
         L.tman_mpgemv_ternary.argtypes = [vp, sz, vp, vp, C.c_float, vp, vp, i, i, i, i, vp, sz, vp]
@@ -218,6 +220,15 @@ def tman_debug_mpgemm_variant(variant, packed, x, y, M, K, N, bits, group, ws, w
                                            packed.numel() * packed.element_size(), _ptr(x), _ptr(y), M, K, N, bits, group,
                                            _ptr(wt), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
            "tman_debug_mpgemm_variant")
+
+
+def tman_debug_role_stamps(ws, ctas, stream=None):
+    """int64 array [ctas][26 warps][4]: wait clocks (two kinds), role clocks, tag; needs the stamps build."""
+    import numpy as np
+    out = np.zeros((ctas, 26, 4), dtype=np.int64)
+    _check(lib().tman_debug_role_stamps(_ptr(ws), ws.numel() * ws.element_size(), ctas, out.ctypes.data, _stream(stream)),
+           "tman_debug_role_stamps")
+    return out
 
 
 def tman_debug_wait_timeout(ws, polls, stream=None) -> None:

@@ -208,6 +208,14 @@ tman_status tman_debug_mpgemm_variant(int variant, const void *packed, size_t pa
                                  reinterpret_cast<cudaStream_t>(stream));
 }
 
+tman_status tman_debug_role_stamps(const void *workspace, size_t ws_bytes, int ctas, long long *out_host, tman_stream_t stream)
+{
+    if (!workspace || !out_host) return TMAN_ERR_NULL;
+    if (!aligned_to(workspace, 256)) return TMAN_ERR_SHAPE;
+    if (ws_bytes < mpgemm_workspace_bytes(1, 128, 8)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return mpgemm_read_stamps(workspace, ctas, out_host, reinterpret_cast<cudaStream_t>(stream));
+}
+
 tman_status tman_debug_indices(const void *packed, int K, int N, int bits, int group,
                                uint8_t *idx, void *workspace, size_t ws_bytes, tman_stream_t stream)
 {

@@ -72,6 +72,19 @@ constexpr size_t kGemmFlagsOff = kWsStatusBytes;
 constexpr size_t kGemmFlags2Off = kWsStatusBytes + 8192;
 constexpr size_t kGemmPartialOff = kGemmFlags2Off + 40960;
 constexpr uint32_t kFlagEmpty = 0x7FA5A5A5u;    // what tman_workspace_init leaves behind
+// Role time stamps (only in a library built with -DTMAN_ROLE_STAMPS; the workspace has room for them in
+// every build so that its layout does not depend on the flag): per CTA and warp four 64-bit words --
+// clocks spent in the role's first kind of wait, in its second kind, in the whole role, and a tag.
+//   warp 0 (TMA producer): waits for a free stage            warp 1 (MMA issuer): accumulator free / stage dequantized
+//   warps 2..17 (dequantization): stage loaded               warps 18..25 (epilogue): accumulators complete
+constexpr int kStampWordsPerWarp = 4;
+constexpr int kGemmWarps = 2 + NUM_DEQ_WARPS + NUM_EPI_WARPS;
+constexpr size_t kStampBytesPerCta = (size_t)kGemmWarps * kStampWordsPerWarp * sizeof(long long);
+#ifdef TMAN_ROLE_STAMPS
+#define TMAN_STAMPED_WAIT(acc, call) ([&]() { const long long t_ = clock64(); const bool r_ = (call); (acc) += clock64() - t_; return r_; }())
+#else
+#define TMAN_STAMPED_WAIT(acc, call) (call)
+#endif
 constexpr size_t kPartialBytesPerCta = (size_t)NUM_EPI_WARPS * 2 * (BN / 64) * CHUNK_BYTES;   // 256 KB, whatever MH
 
 struct GemmParams {
@@ -88,6 +101,7 @@ struct GemmParams {
     int span_tiles;            // the last span_tiles tiles are dealt as equal spans of k-blocks (0: every tile whole)
     int split_s;               // even split: every tile's k-blocks go to split_s workers (0: off)
     int col_fastest;           // tile number = row tile * tiles_n + column tile (else column tile * tiles_m + row tile)
+    long long *stamps;         // role time stamps (written only by a build with TMAN_ROLE_STAMPS)
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -561,6 +575,10 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (tmem_base == 0xFFFFFFFFu) tmem_base = ld_shared_cluster_u32(mapa_u32(smem_u32(tmem_slot), rank ^ 1u));
 
     bool ok = tmem_base != 0xFFFFFFFFu;
+    long long wait_a = 0, wait_b = 0;                  // clocks in this thread's waits (time-stamp builds only)
+#ifdef TMAN_ROLE_STAMPS
+    const long long role_t0 = clock64();
+#endif
     const int worker = (int)blockIdx.x / NCTA, nworkers = (int)gridDim.x / NCTA;
     Span span(p, worker, nworkers);
     Segment sg;
@@ -592,7 +610,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
                     const int s = (int)(it % RING);
                     const uint32_t ph = (it / RING) & 1u;
-                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { ok = false; break; }
+                    if (!TMAN_STAMPED_WAIT(wait_a, mbar_wait(empty0 + 8 * s, ph ^ 1u))) { ok = false; break; }
                     if constexpr (V == kGemmLoadFull) {
                         // the fp16 weight tile itself: this CTA's channels x one k-block, 128-byte swizzle
                         mbar_expect_tx(loaded0 + 8 * s, A_STAGE_BYTES + B_STAGE_BYTES);
@@ -614,13 +632,13 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (lane == 0 && rank == 0) {
             uint32_t it = 0, ti = 0;
             while (ok && span.next(sg)) {
-                if (!mbar_wait(acce, (ti & 1u) ^ 1u)) { ok = false; break; }
+                if (!TMAN_STAMPED_WAIT(wait_a, mbar_wait(acce, (ti & 1u) ^ 1u))) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t idesc = (1u << 4) | ((uint32_t)(tile_bn(sg.tile) >> 3) << 17) | ((uint32_t)((NCTA * BM) >> 4) << 24);
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
                     const int s = (int)(it % RING);
                     const uint32_t ph = (it / RING) & 1u;
-                    if (!mbar_wait(full0 + 8 * s, ph)) { ok = false; break; }
+                    if (!TMAN_STAMPED_WAIT(wait_b, mbar_wait(full0 + 8 * s, ph))) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * B_STAGE_BYTES));
 #pragma unroll
@@ -705,7 +723,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         fetch_sz(Bn, sv_next, zz_next);
                     }
                 }
-                if (!mbar_wait(loaded0 + 8 * s, ph)) { ok = false; break; }
+                if (!TMAN_STAMPED_WAIT(wait_a, mbar_wait(loaded0 + 8 * s, ph))) { ok = false; break; }
                 if (work) {
                     uint32_t w[BITS];
                     const uint32_t pp = p_base + (uint32_t)s * P_STAGE_BYTES;
@@ -761,7 +779,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             int first_w = worker;
             if (!p.split_s && sg.finishes && !sg.whole) first_w = span.owner(sg.tile, 0);
             const int ncontrib = worker - first_w;
-            if (!mbar_wait(accf, ti & 1u)) { ok = false; break; }
+            if (!TMAN_STAMPED_WAIT(wait_a, mbar_wait(accf, ti & 1u))) { ok = false; break; }
             tcgen05_fence_after();
             if (p.split_s) {
                 // ---- even split: the S workers of a tile finish together and share the summing -----------
@@ -997,6 +1015,17 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
 
     if (!ok) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
     tcgen05_fence_before();
+#ifdef TMAN_ROLE_STAMPS
+    if (lane == 0 && p.stamps != nullptr) {
+        long long *st = p.stamps + ((size_t)blockIdx.x * kGemmWarps + warp) * kStampWordsPerWarp;
+        st[0] = wait_a;
+        st[1] = wait_b;
+        st[2] = clock64() - role_t0;
+        st[3] = 0x5354414D50ll;                        // "STAMP": this build writes time stamps
+    }
+#else
+    (void)wait_a; (void)wait_b;
+#endif
     __syncthreads();
     if constexpr (PAIR) cluster_sync_all();            // nobody touches the peer's memory after this
     if (warp == 1 && tmem_base != 0xFFFFFFFFu) {
@@ -1218,7 +1247,23 @@ tman_status mpgemm_plan(int M, int K, int N, int bits, int *out8)
 size_t mpgemm_workspace_bytes(int M, int, int)
 {
     (void)M;
-    return kGemmPartialOff + (size_t)kMaxGemmCtas * kPartialBytesPerCta;
+    return kGemmPartialOff + (size_t)kMaxGemmCtas * (kPartialBytesPerCta + kStampBytesPerCta);
+}
+
+// Copies the role time stamps of the last prefill call out of the workspace (host buffer of
+// ctas x 26 warps x 4 words).  Only a library built with TMAN_ROLE_STAMPS writes them.
+tman_status mpgemm_read_stamps(const void *ws, int ctas, long long *out_host, cudaStream_t s)
+{
+#ifdef TMAN_ROLE_STAMPS
+    if (ctas < 1 || ctas > kMaxGemmCtas) return TMAN_ERR_SHAPE;
+    const uint8_t *src = static_cast<const uint8_t *>(ws) + kGemmPartialOff + (size_t)kMaxGemmCtas * kPartialBytesPerCta;
+    if (cudaMemcpyAsync(out_host, src, (size_t)ctas * kStampBytesPerCta, cudaMemcpyDeviceToHost, s) != cudaSuccess) return TMAN_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return TMAN_ERR_CUDA;
+    return TMAN_OK;
+#else
+    (void)ws; (void)ctas; (void)out_host; (void)s;
+    return TMAN_ERR_UNSUPPORTED;
+#endif
 }
 
 tman_status launch_mpgemm(const void *packed, const void *x, void *y, int M, int K, int N, int bits,
@@ -1300,6 +1345,7 @@ tman_status launch_mpgemm_variant(int variant, const void *packed, const void *x
     p.span_tiles = g.span_tiles;
     p.split_s = g.split_s;
     p.col_fastest = g.col_fastest;
+    p.stamps = reinterpret_cast<long long *>(w8 + kGemmPartialOff + (size_t)kMaxGemmCtas * kPartialBytesPerCta);
     // the fp16 weights [N][K]: boxes of one k-block x a CTA's channels, 128-byte swizzle (the layout the
     // dequantization writes); unused maps are copies of the activation map
     CUtensorMap tmap_wf = tmap_x;

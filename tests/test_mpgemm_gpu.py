@@ -139,6 +139,53 @@ def test_ablation_variants_compute_the_same_numbers(variant, M, K, N, G):
         assert e.value.status in (3, 4)
 
 
+STAMPS_CHILD = """
+import sys, numpy as np, torch
+from paper_2511_11248_b200 import binding as B, helpers as H, synth
+M, K, N, bits, G, out = [int(a) for a in sys.argv[1:6]] + [sys.argv[6]]
+c = synth.small_case(M, K, N, bits, G, seed=M + K + N)
+dev = H.device_case(c)
+packed = H.pack_case(c, dev)
+ws = H.alloc_workspace(B.OP_GEMM, M, K, N, bits, G)
+y = H.alloc_y(M, N)
+B.tman_mpgemm(packed, dev["x"], y, M, K, N, bits, G, ws)
+assert B.tman_read_status(ws) == 0
+H.check_guards()
+plan = B.tman_debug_gemm_plan(M, K, N, bits, G)
+ctas = plan["workers"] * (2 if plan["pair"] else 1)
+np.save(out + ".y.npy", y.cpu().numpy().view(np.uint16))
+np.save(out + ".stamps.npy", B.tman_debug_role_stamps(ws, ctas))
+"""
+
+
+@pytest.mark.parametrize("M,K,N,bits,G", [(1024, 1024, 3560, 4, 128), (300, 8192, 1024, 2, 64)])
+def test_time_stamp_build_computes_the_same_bits(M, K, N, bits, G, tmp_path):
+    # the library built with TMAN_ROLE_STAMPS reads the clock around every role's waits and nothing else:
+    # its output must be bit-identical to the regular library's, and its stamps must be plausible
+    import os
+    import subprocess
+    import sys
+    from paper_2511_11248_b200 import build
+    lib = build.build(stamps=True)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, TMAN_LIBRARY=lib, PYTHONPATH=root)
+    out = str(tmp_path / "stamped")
+    subprocess.run([sys.executable, "-c", STAMPS_CHILD, str(M), str(K), str(N), str(bits), str(G), out],
+                   check=True, env=env, cwd=root, timeout=600)
+    c = synth.small_case(M, K, N, bits, G, seed=M + K + N)
+    want = run_gemm(c).cpu().numpy().view(np.uint16)
+    assert np.array_equal(np.load(out + ".y.npy"), want)
+    st = np.load(out + ".stamps.npy")                  # [ctas][26 warps][wait a, wait b, role, tag]
+    assert np.all(st[:, :, 3] == 0x5354414D50)
+    assert np.all(st[:, :, 2] > 0) and np.all(st[:, :, 0] >= 0) and np.all(st[:, :, 1] >= 0)
+    assert np.all(st[:, :, 0] + st[:, :, 1] <= st[:, :, 2])      # a role cannot wait longer than it lives
+    # the regular library says so when asked for stamps
+    ws = H.alloc_workspace(B.OP_GEMM, M, K, N, bits, G)
+    with pytest.raises(B.TmanError) as e:
+        B.tman_debug_role_stamps(ws, 2)
+    assert e.value.status == 3
+
+
 def test_integer_case_is_exact():
     rng = np.random.default_rng(5)
     c = synth.small_case(130, 512, 136, 3, 64, seed=31)
