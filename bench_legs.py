@@ -371,10 +371,52 @@ def ternary_results(torch, B, H, reps=7):
     return out
 
 
+def ternary_prefill_results(torch, B, H, reps=7):
+    """INT8 prefill on the BitNet sizes: the fused kernel against fp16 torch.matmul on the same shape."""
+    out = []
+    group = 128
+    for M in (128, 1024, 4096):
+        for K, N in ((2560, 2560), (2560, 6912), (6912, 2560), (6912, 6912)):
+            g = torch.Generator(device="cuda")
+            g.manual_seed(M + K + N)
+            codes = torch.randint(0, 3, (K, N), dtype=torch.uint8, device="cuda", generator=g)
+            pk0 = torch.empty(B.tman_packed_bytes(K, N, 2, group), dtype=torch.uint8, device="cuda")
+            B.tman_pack_weights(codes, torch.ones((K // group, N), dtype=torch.float16, device="cuda"),
+                                torch.ones((K // group, N), dtype=torch.uint8, device="cuda"), K, N, 2, group, pk0)
+            ncopy = max(2, int(2.2 * L2_BYTES // pk0.numel()) + 1)
+            pk = [pk0] + [pk0.clone() for _ in range(ncopy - 1)]
+            x = torch.randn((M, K), device="cuda", generator=g).to(torch.float16)
+            a8 = torch.empty((M, K), dtype=torch.int8, device="cuda")
+            sa = torch.empty(max(M, 64), dtype=torch.float32, device="cuda")
+            B.tman_quantize_rows_i8(x, M, K, a8, sa)
+            ys = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in range(2)]
+            ws = workspace(torch, B, B.OP_AUX, 1, K, N, 2, group)
+
+            def run():
+                for i in range(ncopy):
+                    B.tman_mpgemm_ternary_i8(pk[i], a8, sa, 0.02, ys[i % 2], M, K, N, group, ws)
+
+            run()
+            torch.cuda.synchronize()
+            us = event_us(torch, run, reps)[0] / ncopy
+            assert B.tman_read_status(ws) == 0
+            qus = event_us(torch, lambda: B.tman_quantize_rows_i8(x, M, K, a8, sa), reps)[0]
+            del pk
+            torch.cuda.empty_cache()
+            dus = dense_case_us(torch, M, K, N, reps)
+            out.append({"leg": "ternary_prefill", "M": M, "K": K, "N": N, "us": round(us, 1),
+                        "TOPs": round(2.0 * M * K * N / us / 1e6, 1), "quantize_rows_us": round(qus, 1),
+                        "dense_fp16_torch_us": round(dus, 1), "time_vs_dense_fp16": round(us / dus, 2)})
+            torch.cuda.empty_cache()
+    return out
+
+
 def ternary(args, rest=()):
     import torch
     from paper_2511_11248_b200 import binding as B, helpers as H
     for r in ternary_results(torch, B, H):
+        print(json.dumps(r), flush=True)
+    for r in ternary_prefill_results(torch, B, H):
         print(json.dumps(r), flush=True)
 
 

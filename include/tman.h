@@ -163,12 +163,27 @@ tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const i
                                 int M, int K, int N, int group,
                                 void *workspace, size_t ws_bytes, tman_stream_t stream);
 
+/* The same row quantization with 8-bit output (qmax = 127) for the prefill side.  a_i8: int8 [M][K],
+ * 16-byte aligned. */
+tman_status tman_quantize_rows_i8(const void *x_f16, int M, int K, int8_t *a_i8, float *row_scale,
+                                  tman_stream_t stream);
+
+/* Prefill of the integer path (paper Sec. 6.2 "mpGEMM": per-tensor weights are dequantized to INT8 for the
+ * matrix unit; Sec. 4.1 / Fig. 7 two-level lookup; Sec. 4.2 / Fig. 9 three pipelined agents): packed
+ * ternary tiles are staged by TMA, rebuilt as INT8 tiles by bit repacking and a four-entry conversion
+ * table, and multiplied with the 8-bit activations on the tensor cores with 32-bit integer accumulators;
+ *   y[m][n] = fp16( row_scale[m] * w_scale * sum_k a[m][k] * (q[k][n] - 1) ),  M >= 1.
+ * packed: as for tman_mpgemv_ternary.  workspace: at least 256 bytes (status word). */
+tman_status tman_mpgemm_ternary_i8(const void *packed, size_t packed_bytes, const int8_t *a_i8,
+                                   const float *row_scale, float w_scale, void *y_f16, int M, int K, int N,
+                                   int group, void *workspace, size_t ws_bytes, tman_stream_t stream);
+
 /* Prefill side of the integer path, the dequantization step alone (paper Sec. 6.2 "mpGEMM": per-tensor
  * weights are dequantized to INT8 for the matrix unit; Sec. 4.1 / Fig. 7: by two table lookups, bit
  * repacking and a conversion table, here with the INT8 values -1, 0, +1 as the table's entries).
  * w8_nk: output, int8 [N][K] (channel-major, 16-byte aligned).  workspace: at least 256 bytes (status
- * word: a header that does not match leaves the output untouched).  The INT8 matrix multiplication that
- * would consume these tiles on the tensor cores is not part of the library. */
+ * word: a header that does not match leaves the output untouched).  tman_mpgemm_ternary_i8 does the same
+ * lookups inside its pipeline; this call exists to check them bit for bit and to time them alone. */
 tman_status tman_dequant_ternary_int8(const void *packed, size_t packed_bytes, int K, int N, int group,
                                       int8_t *w8_nk, void *workspace, size_t ws_bytes, tman_stream_t stream);
 

@@ -70,6 +70,7 @@ void oracle_quantize_rows(const uint16_t *x, int M, int K, int qmax, int32_t *a,
 void oracle_ternary_matmul(const int32_t *a, const uint8_t *q, int M, int K, int N, int64_t *acc)
 {
     int m, n, k;
+#pragma omp parallel for private(n, k) schedule(static)
     for (m = 0; m < M; ++m)
         for (n = 0; n < N; ++n) {
             int64_t s = 0;
@@ -137,6 +138,7 @@ void oracle_ternary_dequant_int8(const uint8_t *q, int K, int N, int8_t *w8)
 void oracle_int8_matmul(const int32_t *a8, const int8_t *w8, int M, int K, int N, int64_t *acc)
 {
     int m, n, k;
+#pragma omp parallel for private(n, k) schedule(static)
     for (m = 0; m < M; ++m)
         for (n = 0; n < N; ++n) {
             int64_t s = 0;

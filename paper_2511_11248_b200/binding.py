@@ -24,7 +24,7 @@ EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",
     "tman_workspace_init", "tman_read_status", "tman_pack_weights", "tman_unpack_weights",
     "tman_mpgemv", "tman_mpgemm", "tman_debug_indices", "tman_debug_luts", "tman_debug_gemm_plan", "tman_mpgemv_static", "tman_mpgemv_grouped",
-    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for", "tman_debug_gemv_plan", "tman_debug_wait_timeout", "tman_debug_mpgemm_variant", "tman_quantize_rows", "tman_mpgemv_ternary", "tman_dequant_ternary_int8", "tman_debug_role_stamps",
+    "tman_debug_microbench", "tman_debug_cluster_capacity", "tman_debug_gemm_plan_for", "tman_debug_gemv_plan", "tman_debug_wait_timeout", "tman_debug_mpgemm_variant", "tman_quantize_rows", "tman_mpgemv_ternary", "tman_dequant_ternary_int8", "tman_debug_role_stamps", "tman_quantize_rows_i8", "tman_mpgemm_ternary_i8",
 ]
 
 _lib = None
@@ -67,6 +67,8 @@ def lib() -> C.CDLL:
         L.tman_debug_gemm_plan_for.argtypes = [i, i, i, i, i, i, i, C.POINTER(C.c_int)]
         L.tman_debug_gemv_plan.argtypes = [i, i, i, i, i, i, sz, C.POINTER(C.c_int)]
         L.tman_debug_wait_timeout.argtypes = [vp, sz, C.c_uint, vp]
+        L.tman_quantize_rows_i8.argtypes = [vp, i, i, vp, vp, vp]
+        L.tman_mpgemm_ternary_i8.argtypes = [vp, sz, vp, vp, C.c_float, vp, i, i, i, i, vp, sz, vp]
         L.tman_debug_role_stamps.argtypes = [vp, sz, i, vp, vp]
         L.tman_dequant_ternary_int8.argtypes = [vp, sz, i, i, i, vp, vp, sz, vp]
         L.tman_quantize_rows.argtypes = [vp, i, i, i, vp, vp, vp]
@@ -200,6 +202,16 @@ def tman_dequant_ternary_int8(packed, K, N, group, w8, ws, stream=None) -> None:
     _check(lib().tman_dequant_ternary_int8(_ptr(packed), packed.numel() * packed.element_size(), K, N, group, _ptr(w8),
                                            _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
            "tman_dequant_ternary_int8")
+
+
+def tman_quantize_rows_i8(x, M, K, a, row_scale, stream=None) -> None:
+    _check(lib().tman_quantize_rows_i8(_ptr(x), M, K, _ptr(a), _ptr(row_scale), _stream(stream)), "tman_quantize_rows_i8")
+
+
+def tman_mpgemm_ternary_i8(packed, a, row_scale, w_scale, y, M, K, N, group, ws, stream=None) -> None:
+    _check(lib().tman_mpgemm_ternary_i8(_ptr(packed), packed.numel() * packed.element_size(), _ptr(a), _ptr(row_scale),
+                                        float(w_scale), _ptr(y), M, K, N, group, _ptr(ws), ws.numel() * ws.element_size(),
+                                        _stream(stream)), "tman_mpgemm_ternary_i8")
 
 
 def tman_quantize_rows(x, M, K, qmax, a, row_scale, stream=None) -> None:

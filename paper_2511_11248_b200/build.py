@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtman.so")
 LIB_STAMPS = os.path.join(HERE, "libtman_stamps.so")   # the same library with role time stamps in the prefill kernel
-SOURCES = ["api.cu", "pack.cu", "mpgemv.cu", "mpgemv_static.cu", "mpgemm.cu", "microbench.cu"]
+SOURCES = ["api.cu", "pack.cu", "mpgemv.cu", "mpgemv_static.cu", "mpgemm.cu", "mpgemm_i8.cu", "microbench.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "--shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,

@@ -173,6 +173,26 @@ tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const i
                                  reinterpret_cast<cudaStream_t>(stream));
 }
 
+tman_status tman_quantize_rows_i8(const void *x_f16, int M, int K, int8_t *a_i8, float *row_scale, tman_stream_t stream)
+{
+    if (!x_f16 || !a_i8 || !row_scale) return TMAN_ERR_NULL;
+    if (M < 1 || K < 1) return TMAN_ERR_SHAPE;
+    return launch_quantize_rows_i8(x_f16, M, K, a_i8, row_scale, reinterpret_cast<cudaStream_t>(stream));
+}
+
+tman_status tman_mpgemm_ternary_i8(const void *packed, size_t packed_bytes, const int8_t *a_i8, const float *row_scale,
+                                   float w_scale, void *y_f16, int M, int K, int N, int group,
+                                   void *workspace, size_t ws_bytes, tman_stream_t stream)
+{
+    tman_status st = check_matmul(packed, packed_bytes, a_i8, y_f16, M, K, N, 2, group, workspace);
+    if (st != TMAN_OK) return st;
+    if (!row_scale) return TMAN_ERR_NULL;
+    if (K > (1 << 24)) return TMAN_ERR_UNSUPPORTED;             // K * 127 must fit the 32-bit accumulators
+    if (ws_bytes < kWsStatusBytes) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_mpgemm_ternary_i8(packed, a_i8, row_scale, w_scale, y_f16, M, K, N, group, workspace,
+                                    reinterpret_cast<cudaStream_t>(stream));
+}
+
 tman_status tman_dequant_ternary_int8(const void *packed, size_t packed_bytes, int K, int N, int group, int8_t *w8_nk,
                                       void *workspace, size_t ws_bytes, tman_stream_t stream)
 {

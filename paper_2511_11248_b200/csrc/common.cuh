@@ -139,6 +139,9 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
 size_t      mpgemm_workspace_bytes(int M, int K, int N);
 tman_status mpgemm_plan(int M, int K, int N, int bits, int *out8);
 tman_status mpgemm_plan_for(int M, int K, int N, int bits, int sms, int resident, int *out8);
+tman_status launch_quantize_rows_i8(const void *x, int M, int K, int8_t *a, float *s_a, cudaStream_t s);
+tman_status launch_mpgemm_ternary_i8(const void *packed, const int8_t *a8, const float *row_scale, float w_scale, void *y,
+                                     int M, int K, int N, int group, void *ws, cudaStream_t s);
 tman_status mpgemm_read_stamps(const void *ws, int ctas, long long *out_host, cudaStream_t s);
 tman_status launch_mpgemm_variant(int variant, const void *packed, const void *x, void *y, int M, int K, int N, int bits,
                                   int group, const void *wt_f16, void *ws, size_t ws_bytes, cudaStream_t s);

@@ -123,3 +123,39 @@ def test_int8_dequantization_is_bit_exact(K, N, group):
     other = pack_ternary(np.ones((K, N + 8), dtype=np.uint8), group)
     B.tman_dequant_ternary_int8(other, K, N, group, w8, ws)
     assert B.tman_read_status(ws) == 5 and bool((w8 == 55).all())
+
+
+# one tile, ragged tokens and channels, several k-blocks and tiles per CTA, the paper's BitNet sizes
+I8_SHAPES = [(128, 128, 128, 128), (1, 256, 8, 64), (100, 384, 136, 128), (300, 1024, 264, 32), (513, 2560, 2560, 128),
+             (1024, 6912, 2560, 128), (2048, 2560, 6912, 64)]
+
+
+@pytest.mark.parametrize("M,K,N,group", I8_SHAPES)
+def test_int8_prefill_matches_the_integer_oracle(M, K, N, group):
+    x, t, q, s_w = ternary_case(M, K, N, seed=M + K + N, spread=2.0)
+    s_w32 = float(np.float32(s_w))
+    a_ref, s_ref = oi.quantize_rows(x, 127)
+    y_ref = oi.scale_result(oi.int8_matmul(a_ref, oi.ternary_dequant_int8(q)), s_ref, s_w32)
+
+    packed = pack_ternary(q, group)
+    xd = torch.from_numpy(x.view(np.int16)).cuda().view(torch.float16)
+    a8 = H.guarded_bytes(M * K, "a_i8").view(torch.int8).view(M, K)
+    s = H.guarded_bytes(((M * 4 + 255) // 256) * 256, "row_scale").view(torch.float32)
+    B.tman_quantize_rows_i8(xd, M, K, a8, s)
+    torch.cuda.synchronize()
+    assert np.array_equal(a8.cpu().numpy().astype(np.int32), a_ref)                   # integers: bit-exact
+    assert np.array_equal(s[:M].cpu().numpy().astype(np.float64), s_ref)
+    ws = H.alloc_workspace(B.OP_AUX, 1, K, N, 2, group)
+    y = H.alloc_y(M, N)
+    for _ in range(2):
+        B.tman_mpgemm_ternary_i8(packed, a8, s, s_w, y, M, K, N, group, ws)
+        assert B.tman_read_status(ws) == 0
+        H.check_guards()
+        got = H.to_f64(y)
+        assert np.all(np.isfinite(got))
+        # exact integer sums; one fp32 product of scales, one fp32 product with the sum, one rounding to fp16
+        assert np.all(np.abs(got - y_ref) <= np.abs(y_ref) * 2.0 ** -10 + 1e-7)
+    # a buffer with another header is refused, the output stays
+    y.fill_(3.0)
+    B.tman_mpgemm_ternary_i8(torch.zeros_like(packed), a8, s, s_w, y, M, K, N, group, ws)
+    assert B.tman_read_status(ws) == 5 and bool((y == 3.0).all())
