@@ -8,7 +8,7 @@
 //
 // One CTA per SM walks over 128-token x 128-channel tiles.  Per k-block of 128 (one 128-byte row of INT8):
 //   warp 0      TMA: the activation tile (2-D map, 128-byte swizzle) and the two plane tiles of the
-//               CTA's channels (3-D map over (word/column, plane, strip)) into a 3-stage ring
+//               CTA's channels (3-D map over (word/column, plane, strip)) into a 6-stage ring
 //   warps 2-5   dequantization: a thread takes the plane words of one strip (four channels) and 32 k:
 //               level 1 interleaves the two planes into 2-bit codes, one per nibble, in k order; level 2
 //               looks four codes at a time up in a four-entry byte table {-1, 0, +1, 0} with one byte
@@ -27,7 +27,7 @@ namespace tman {
 namespace {
 
 constexpr int I8_BM = 128, I8_BN = 128, I8_BK = 128;
-constexpr int I8_STAGES = 3;
+constexpr int I8_STAGES = 6;                                            // 36 KB each: loads of six k-blocks in flight
 constexpr int I8_A_BYTES = I8_BM * I8_BK;                               // 16 KB
 constexpr int I8_B_BYTES = I8_BN * I8_BK;                               // 16 KB
 constexpr int I8_P_PLANE_BYTES = (I8_BN / 4) * (I8_BK / 32) * 16;       // 32 strips x 4 words x 4 columns x 4 B
