@@ -148,7 +148,8 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed /*host*/, c
 
 /* Per-row symmetric quantization of activations: row_scale[m] = max_k |x[m][k]| / qmax (1 for a row of
  * zeros), a[m][k] = round(x[m][k] / row_scale[m]) clamped to +-qmax; division and rounding (to nearest
- * even) in single precision.  qmax = 32767 (decode) or 127.  a_i16: int16 [M][K]; row_scale: fp32 [M]. */
+ * even) in single precision.  qmax = 32767 (decode) or 127.  a_i16: int16 [M][K]; row_scale: fp32 [M].
+ * x_f16 and a_i16 are 16-byte aligned (TMAN_ERR_SHAPE otherwise). */
 tman_status tman_quantize_rows(const void *x_f16, int M, int K, int qmax, int16_t *a_i16, float *row_scale,
                                tman_stream_t stream);
 

@@ -177,6 +177,7 @@ tman_status tman_quantize_rows_i8(const void *x_f16, int M, int K, int8_t *a_i8,
 {
     if (!x_f16 || !a_i8 || !row_scale) return TMAN_ERR_NULL;
     if (M < 1 || K < 1) return TMAN_ERR_SHAPE;
+    if (!matrices_aligned(x_f16, a_i8)) return TMAN_ERR_SHAPE;
     return launch_quantize_rows_i8(x_f16, M, K, a_i8, row_scale, reinterpret_cast<cudaStream_t>(stream));
 }
 

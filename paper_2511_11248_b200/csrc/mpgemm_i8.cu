@@ -224,40 +224,7 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 }
 
-// Row quantization with INT8 output (see quantize_rows_kernel in mpgemv.cu for the 16-bit one): the same
-// arithmetic, single-precision division and rounding to nearest even.
-__global__ void __launch_bounds__(1024) quantize_rows_i8_kernel(const __half *__restrict__ x, int K, int8_t *__restrict__ a,
-                                                                float *__restrict__ s_a)
-{
-    __shared__ float red[32];
-    const __half *row = x + (size_t)blockIdx.x * K;
-    float amax = 0.f;
-    for (int k = threadIdx.x; k < K; k += blockDim.x) amax = fmaxf(amax, fabsf(__half2float(row[k])));
-    for (int mask = 16; mask > 0; mask >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, mask));
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
-        for (int mask = 16; mask > 0; mask >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, mask));
-        if (threadIdx.x == 0) red[0] = v;
-    }
-    __syncthreads();
-    amax = red[0];
-    const float scale = amax > 0.f ? __fdiv_rn(amax, 127.f) : 1.f;
-    if (threadIdx.x == 0) s_a[blockIdx.x] = scale;
-    for (int k = threadIdx.x; k < K; k += blockDim.x) {
-        const int r = __float2int_rn(__fdiv_rn(__half2float(row[k]), scale));
-        a[(size_t)blockIdx.x * K + k] = (int8_t)max(-127, min(127, r));
-    }
-}
-
 }  // namespace
-
-tman_status launch_quantize_rows_i8(const void *x, int M, int K, int8_t *a, float *s_a, cudaStream_t s)
-{
-    quantize_rows_i8_kernel<<<(unsigned)M, 256, 0, s>>>(static_cast<const __half *>(x), K, a, s_a);
-    return launch_status();
-}
 
 tman_status launch_mpgemm_ternary_i8(const void *packed, const int8_t *a8, const float *row_scale, float w_scale, void *y,
                                      int M, int K, int N, int group, void *ws, cudaStream_t s)

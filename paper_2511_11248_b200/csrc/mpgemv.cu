@@ -1000,12 +1000,13 @@ tman_status launch_mpgemv_grouped(int count, const void *const *packed, const vo
 // Per-row symmetric quantization of the activations (paper Sec. 6.1, A_INT16; 8 bits for the matrix unit):
 // s_a = max|x| / qmax and a = round(x / s_a), both in single precision with correctly rounded division and
 // rounding to nearest even, so that the integers are the same on any IEEE machine.  One CTA per row.
+template <typename OUT>      // int16_t or int8_t
 __global__ void __launch_bounds__(1024) quantize_rows_kernel(const __half *__restrict__ x, int K, int qmax,
-                                                             int16_t *__restrict__ a, float *__restrict__ s_a)
+                                                             OUT *__restrict__ a, float *__restrict__ s_a)
 {
     __shared__ float red[32];
     const __half *row = x + (size_t)blockIdx.x * K;
-    int16_t *out = a + (size_t)blockIdx.x * K;
+    OUT *out = a + (size_t)blockIdx.x * K;
     // eight values per thread and step when the row allows 16-byte accesses (K % 8 == 0, checked by the host)
     const bool vec = (K & 7) == 0;
     const int nvec = vec ? K >> 3 : 0;
@@ -1036,20 +1037,36 @@ __global__ void __launch_bounds__(1024) quantize_rows_kernel(const __half *__res
     for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
         const uint4 q = __ldg(reinterpret_cast<const uint4 *>(row) + i);        // second read: from L1/L2
         const __half *h = reinterpret_cast<const __half *>(&q);
-        uint4 o;
-        o.x = (uint32_t)(quant(h[0]) & 0xFFFF) | ((uint32_t)quant(h[1]) << 16);
-        o.y = (uint32_t)(quant(h[2]) & 0xFFFF) | ((uint32_t)quant(h[3]) << 16);
-        o.z = (uint32_t)(quant(h[4]) & 0xFFFF) | ((uint32_t)quant(h[5]) << 16);
-        o.w = (uint32_t)(quant(h[6]) & 0xFFFF) | ((uint32_t)quant(h[7]) << 16);
-        reinterpret_cast<uint4 *>(out)[i] = o;
+        if constexpr (sizeof(OUT) == 2) {
+            uint4 o;
+            o.x = (uint32_t)(quant(h[0]) & 0xFFFF) | ((uint32_t)quant(h[1]) << 16);
+            o.y = (uint32_t)(quant(h[2]) & 0xFFFF) | ((uint32_t)quant(h[3]) << 16);
+            o.z = (uint32_t)(quant(h[4]) & 0xFFFF) | ((uint32_t)quant(h[5]) << 16);
+            o.w = (uint32_t)(quant(h[6]) & 0xFFFF) | ((uint32_t)quant(h[7]) << 16);
+            reinterpret_cast<uint4 *>(out)[i] = o;
+        } else {
+            uint2 o;
+            o.x = (uint32_t)(quant(h[0]) & 0xFF) | ((uint32_t)(quant(h[1]) & 0xFF) << 8) |
+                  ((uint32_t)(quant(h[2]) & 0xFF) << 16) | ((uint32_t)quant(h[3]) << 24);
+            o.y = (uint32_t)(quant(h[4]) & 0xFF) | ((uint32_t)(quant(h[5]) & 0xFF) << 8) |
+                  ((uint32_t)(quant(h[6]) & 0xFF) << 16) | ((uint32_t)quant(h[7]) << 24);
+            reinterpret_cast<uint2 *>(out)[i] = o;
+        }
     }
-    for (int k = 8 * nvec + threadIdx.x; k < K; k += blockDim.x) out[k] = (int16_t)quant(row[k]);
+    for (int k = 8 * nvec + threadIdx.x; k < K; k += blockDim.x) out[k] = (OUT)quant(row[k]);
 }
 
 tman_status launch_quantize_rows(const void *x, int M, int K, int qmax, int16_t *a, float *s_a, cudaStream_t s)
 {
     const int threads = K >= 8192 ? 1024 : (K >= 2048 ? 512 : 256);
-    quantize_rows_kernel<<<(unsigned)M, threads, 0, s>>>(static_cast<const __half *>(x), K, qmax, a, s_a);
+    quantize_rows_kernel<int16_t><<<(unsigned)M, threads, 0, s>>>(static_cast<const __half *>(x), K, qmax, a, s_a);
+    return launch_status();
+}
+
+tman_status launch_quantize_rows_i8(const void *x, int M, int K, int8_t *a, float *s_a, cudaStream_t s)
+{
+    const int threads = K >= 8192 ? 1024 : (K >= 2048 ? 512 : 256);
+    quantize_rows_kernel<int8_t><<<(unsigned)M, threads, 0, s>>>(static_cast<const __half *>(x), K, 127, a, s_a);
     return launch_status();
 }
 
