@@ -221,15 +221,32 @@ def config3_results(torch, B, H, reps=7, dense=False, bits_list=(2, 3, 4), Ms=(1
     return out
 
 
+def config3_projection_results(torch, B, H, reps=7, bits_list=(2, 3, 4), Ms=(1, 2, 4, 8)):
+    """Each of the seven projections alone (one call per projection, rotating copies larger than L2)."""
+    out = []
+    for bits in bits_list:
+        for M in Ms:
+            for name, K, N in LLAMA3_8B_LAYER:
+                med, best, nbytes, nsets = decode_calls_us(torch, B, H, M, bits, 128, [[(K, N)]], reps)
+                out.append({"leg": "config3_projection", "proj": name, "M": M, "K": K, "N": N, "bits": bits, "group": 128,
+                            "us": round(med, 2), "us_best": round(best, 2), "weight_stream_GBs": round(nbytes / med / 1e3, 1)})
+                torch.cuda.empty_cache()
+    return out
+
+
 def config3(args, rest=()):
     import torch
     from paper_2511_11248_b200 import binding as B, helpers as H
     ap = argparse.ArgumentParser(prog="bench.py --leg config3")
     ap.add_argument("--dense", action="store_true")
+    ap.add_argument("--per-projection", action="store_true", help="also time each of the seven projections alone")
     ap.add_argument("--reps", type=int, default=7)
     a = ap.parse_args(list(rest))
     for r in config3_results(torch, B, H, a.reps, a.dense):
         print(json.dumps(r), flush=True)
+    if a.per_projection:
+        for r in config3_projection_results(torch, B, H, a.reps):
+            print(json.dumps(r), flush=True)
 
 
 # ---- prefill shape sweep (config 5) --------------------------------------------------------------------
