@@ -1,8 +1,9 @@
 // Decode path: bit-serial table-lookup mpGEMV (paper Sec. 2.2 "Bit-serial table lookup", Fig. 2;
 // Sec. 4.3 "Mapping of LUT-based Decoding").
 //
-// Work split.  The reduction dimension is cut into K-slices of 32/MT plane words (MT = number
-// of activation rows a table entry carries).  One CTA owns one K-slice: it builds that slice's
+// Work split.  The reduction dimension is cut into K-slices of 8 to 32 plane words (16 for one
+// activation row; 32, 16, 8 for 2, 3-4, 5-8 rows, whose table entries carry the rows as fp16 pairs).  One
+// CTA owns one K-slice: it builds that slice's
 // activation tables in shared memory once and reuses them for every output column it visits
 // (the paper's "maximise reuse of cached lookup tables").  Inside a warp a lane owns ONE plane
 // word, i.e. 32 consecutive activations = four 8-activation table groups, and one shared-memory
@@ -22,8 +23,8 @@
 // "ready" flag, so no fence and no counter sits between the last lookup and the output; the poll
 // is bounded and reports TMAN_ERR_TIMEOUT.
 //
-// Streaming.  A warp works through units (a few strips of four columns).  With one activation row
-// every strip's registers are refilled with the next unit's strip as soon as its lookups are done;
+// Streaming.  A warp works through units (a few strips of four columns).  With up to four activation
+// rows every strip's registers are refilled with the next unit's strip as soon as its lookups are done;
 // with more rows the next unit sits in a second set of registers.  Either way HBM reads overlap the
 // lookups.  The first
 // loads (header words, first unit) are issued before the kernel waits for the previous kernel in
