@@ -414,25 +414,37 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 reinterpret_cast<float *>(smem + kGemvTableBytes)[2 * mb + r] = __uint_as_float(e << 23);
         }
         {
-            const int ph = warp;
+            // warp w fills, for index byte c = w % 4 of the word, the entries whose high index nibble is
+            // 4 * (w / 4) .. 4 * (w / 4) + 3: the low-nibble sums of a byte are then computed once per warp
+            const int c = warp & 3;
+            float lo[2][16], xh[2][4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                float lo[2][16], hi[2];
+            for (int r = 0; r < 2; ++r) {
+                float xv[8];
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    // the c-th half2 of quarter qq: four-way select on the warp-uniform c
+                    const uint4 q4 = xraw[r][qq];
+                    const uint32_t u = c == 0 ? q4.x : c == 1 ? q4.y : c == 2 ? q4.z : q4.w;
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&u));
+                    xv[qq] = f.x * inv[r];
+                    xv[qq + 4] = f.y * inv[r];
+                }
+                lut16(xv[0], xv[1], xv[2], xv[3], lo[r]);
+#pragma unroll
+                for (int qq = 0; qq < 4; ++qq) xh[r][qq] = xv[4 + qq];
+            }
+#pragma unroll
+            for (int pq = 0; pq < 4; ++pq) {
+                const int ph = 4 * (warp >> 2) + pq;
+                float hi[2];
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
-                    float xv[8];
-#pragma unroll
-                    for (int qq = 0; qq < 4; ++qq) {
-                        const float2 f = __half22float2(reinterpret_cast<const __half2 *>(&xraw[r][qq])[c]);
-                        xv[qq] = f.x * inv[r];
-                        xv[qq + 4] = f.y * inv[r];
-                    }
-                    lut16(xv[0], xv[1], xv[2], xv[3], lo[r]);
                     hi[r] = 0.f;
-                    if (ph & 1) hi[r] += xv[4];
-                    if (ph & 2) hi[r] += xv[5];
-                    if (ph & 4) hi[r] += xv[6];
-                    if (ph & 8) hi[r] += xv[7];
+                    if (ph & 1) hi[r] += xh[r][0];
+                    if (ph & 2) hi[r] += xh[r][1];
+                    if (ph & 4) hi[r] += xh[r][2];
+                    if (ph & 8) hi[r] += xh[r][3];
                 }
                 uint8_t *dst = smem + table_imm(c) + (uint32_t)(ph * 16) * 256u + (uint32_t)lane * 4u;
 #pragma unroll
