@@ -817,9 +817,9 @@ static tman_status launch_one(GemvParams p, int sms, cudaStream_t s)
 template <int BITS, int MT, int PRE, int HR>
 static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
 {
-    // one row: fp32 tables over half-warp slices, large units on one rolling set of registers;
-    // more rows: fp16 row pairs, small double-buffered units
-    constexpr int ROLL = (HR && MT == 4) ? 0 : 1;
+    // one row: fp32 tables over half-warp slices, large units; more rows: fp16 row pairs, smaller units
+    // (measured: 2 strips per unit for up to four rows, 1 for eight).  All on one rolling set of registers.
+    constexpr int ROLL = 1;
     constexpr int S = (HR && MT == 4) ? 1 : (HR && MT == 2) ? 2 : ((BITS == 2) ? 4 : 2);
     constexpr int HALF = HR ? 0 : 1;
     if (p.count > 1) return launch_one<BITS, MT, S, PRE, HALF, 1, ROLL, HR>(p, sms, s);
@@ -831,15 +831,15 @@ static tman_status launch_mt(GemvParams p, int sms, cudaStream_t s)
 // words; its table entries have `slots` 32-bit slots (one fp32 row, or two fp16 rows each).  The time of a
 // pass is modelled as fixed + per_mb x megabytes of bit planes; the constants were fitted to calls timed
 // in a CUDA graph on a B200 (K = 4096, N = 14336; 2- and 4-bit for one row, 4-bit for the others):
-//   rows 1: 6.9 / 9.7 us   rows 2: 11.4 us   rows 4: 15.3 us   rows 8: 25.6 us.
+//   rows 1: 6.9 / 9.7 us   rows 2: 10.7 us   rows 4: 14.9 us   rows 8: 23.6 us.
 // The slope grows with the rows because an entry of 2 / 4 / 8 fp16 rows takes 1 / 2 / 4 shared-memory
 // wavefronts per lookup.
 struct GemvVariant { int rows, words, slots, half_slices; double fixed_us, us_per_mb; };
 static const GemvVariant kGemvVariants[kGemvVariantCount] = {
     {1, 16, 1, 1, 4.10, 0.190},
-    {2, 32, 1, 0, 4.35, 0.240},
-    {4, 16, 2, 0, 4.85, 0.355},
-    {8, 8, 4, 0, 5.85, 0.670},
+    {2, 32, 1, 0, 4.35, 0.216},
+    {4, 16, 2, 0, 4.85, 0.341},
+    {8, 8, 4, 0, 5.85, 0.605},
 };
 
 static size_t variant_ws_bytes(const GemvVariant &v, int K, int N)
