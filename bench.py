@@ -442,11 +442,11 @@ def run_ours(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under
-# profiles/.  mpGEMV: one gate/up-sized launch moved 17.03 MB for 16.78 MB of algorithmic bytes
-# (+1.5 %); traffic grows with the bytes streamed, so the step's mean launch (25.17 MB) is scaled
+# profiles/.  mpGEMV: one gate/up-sized launch moved 17.04 MB for 16.78 MB of algorithmic bytes
+# (+1.5 %; counters re-taken on the present kernel build); traffic grows with the bytes streamed, so the step's mean launch (25.17 MB) is scaled
 # by the same ratio.  mpGEMM: the M=1024, K=4096, N=14336 launch (the larger of the two timed shapes)
 # read 39.2 MB and wrote 0.4 - 2.5 MB (the output mostly stays in L2).
-TRAFFIC_BYTES_PER_LAUNCH = 25171968.0 * (17.03 / 16.78)
+TRAFFIC_BYTES_PER_LAUNCH = 25171968.0 * (17.04 / 16.78)
 GEMM_TRAFFIC_BYTES_PER_LAUNCH = 40.6e6
 
 
