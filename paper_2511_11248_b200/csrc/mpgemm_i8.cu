@@ -6,15 +6,16 @@
 //   acc[m][n] = sum_k a8[m][k] * (q[k][n] - 1)        (exact, int32 accumulators in tensor memory)
 //   y[m][n]   = fp16( row_scale[m] * w_scale * acc[m][n] )
 //
-// One CTA per SM walks over 128-token x 128-channel tiles.  Per k-block of 128 (one 128-byte row of INT8):
+// One CTA per SM walks over tiles of 128 tokens x BN channels (BN = 256 when the output still has two
+// tiles or more per SM, else 128).  Per k-block of 128 (one 128-byte row of INT8):
 //   warp 0      TMA: the activation tile (2-D map, 128-byte swizzle) and the two plane tiles of the
-//               CTA's channels (3-D map over (word/column, plane, strip)) into a 6-stage ring
-//   warps 2-5   dequantization: a thread takes the plane words of one strip (four channels) and 32 k:
+//               CTA's channels (3-D map over (word/column, plane, strip)) into a ring of 6 (BN = 128) or 4 stages
+//   next BN/32 warps   dequantization: a thread takes the plane words of one strip (four channels) and 32 k:
 //               level 1 interleaves the two planes into 2-bit codes, one per nibble, in k order; level 2
 //               looks four codes at a time up in a four-entry byte table {-1, 0, +1, 0} with one byte
 //               permute; 32 INT8 per channel are stored into the K-major, 128-byte-swizzled weight tile
-//   warp 1      tcgen05.mma kind::i8 (128 x 128 x 32 per instruction), commit releases the stage
-//   warps 6-9   epilogue: tcgen05.ld of 32 tokens x 32 channels, integer -> float, the row's and the
+//   warp 1      tcgen05.mma kind::i8 (128 x BN x 32 per instruction), commit releases the stage
+//   last 4 warps   epilogue: tcgen05.ld of 32 tokens x 32 channels, integer -> float, the row's and the
 //               tensor's scale, fp16, 64-byte row stores
 // Every wait is bounded (about a second) and reports TMAN_ERR_TIMEOUT; tensor memory is always freed.
 #include "common.cuh"
@@ -26,16 +27,20 @@
 namespace tman {
 namespace {
 
-constexpr int I8_BM = 128, I8_BN = 128, I8_BK = 128;
-constexpr int I8_STAGES = 6;                                            // 36 KB each: loads of six k-blocks in flight
+constexpr int I8_BM = 128, I8_BK = 128;
 constexpr int I8_A_BYTES = I8_BM * I8_BK;                               // 16 KB
-constexpr int I8_B_BYTES = I8_BN * I8_BK;                               // 16 KB
-constexpr int I8_P_PLANE_BYTES = (I8_BN / 4) * (I8_BK / 32) * 16;       // 32 strips x 4 words x 4 columns x 4 B
-constexpr int I8_P_BYTES = 2 * I8_P_PLANE_BYTES;
-constexpr int I8_DEQ_WARPS = 4, I8_EPI_WARPS = 4;
-constexpr int I8_THREADS = 32 * (2 + I8_DEQ_WARPS + I8_EPI_WARPS);
-constexpr int I8_TMEM_COLS = I8_BN;
-constexpr int I8_SMEM_BYTES = I8_STAGES * (I8_A_BYTES + I8_B_BYTES + I8_P_BYTES) + 256;
+constexpr int I8_EPI_WARPS = 4;
+// Tile width BN = 128 or 256 channels (256 when the output still has enough tiles for every SM): one
+// dequantization warp per 32 channels, as many stages as fit the shared memory.
+template <int BN> struct I8Cfg {
+    static constexpr int B_BYTES = BN * I8_BK;                              // 16 / 32 KB
+    static constexpr int P_PLANE_BYTES = (BN / 4) * (I8_BK / 32) * 16;      // strips x 4 words x 4 columns x 4 B
+    static constexpr int P_BYTES = 2 * P_PLANE_BYTES;
+    static constexpr int STAGES = BN == 128 ? 6 : 4;                        // 36 / 56 KB each
+    static constexpr int DEQ_WARPS = BN / 32;
+    static constexpr int THREADS = 32 * (2 + DEQ_WARPS + I8_EPI_WARPS);
+    static constexpr int SMEM_BYTES = STAGES * (I8_A_BYTES + B_BYTES + P_BYTES) + 256;
+};
 
 struct GemmI8Params {
     const uint8_t *packed;
@@ -47,9 +52,13 @@ struct GemmI8Params {
     int tiles_m, tiles_n;
 };
 
-__global__ void __launch_bounds__(I8_THREADS, 1)
+template <int I8_BN>
+__global__ void __launch_bounds__(I8Cfg<I8_BN>::THREADS, 1)
 mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w, const GemmI8Params p)
 {
+    using C = I8Cfg<I8_BN>;
+    constexpr int I8_STAGES = C::STAGES, I8_B_BYTES = C::B_BYTES, I8_P_PLANE_BYTES = C::P_PLANE_BYTES, I8_P_BYTES = C::P_BYTES;
+    constexpr int I8_DEQ_WARPS = C::DEQ_WARPS, I8_TMEM_COLS = I8_BN;
     extern __shared__ __align__(1024) uint8_t smem[];
     if (!header_matches(p.packed, p.K, p.N, 2, p.group)) {          // same answer in every CTA
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
@@ -116,7 +125,7 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            // instruction descriptor: D = s32, A = B = s8, both K-major, N = 128, M = 128
+            // instruction descriptor: D = s32, A = B = s8, both K-major, N = tile width, M = 128
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(I8_BN >> 3) << 17) | ((uint32_t)(I8_BM >> 4) << 24);
             uint32_t it = 0, ti = 0;
             for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
@@ -226,6 +235,21 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
 }  // namespace
 
+namespace {
+template <int BN>
+tman_status launch_i8(const CUtensorMap &tmap_a, const CUtensorMap &tmap_w, GemmI8Params p, int sms, cudaStream_t s)
+{
+    using C = I8Cfg<BN>;
+    p.tiles_n = (p.N + BN - 1) / BN;
+    const int tiles = p.tiles_m * p.tiles_n;
+    auto kern = mpgemm_i8_kernel<BN>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) return TMAN_ERR_CUDA;
+    const int grid = tiles < sms ? tiles : sms;
+    kern<<<(unsigned)grid, C::THREADS, C::SMEM_BYTES, s>>>(tmap_a, tmap_w, p);
+    return launch_status();
+}
+}  // namespace
+
 tman_status launch_mpgemm_ternary_i8(const void *packed, const int8_t *a8, const float *row_scale, float w_scale, void *y,
                                      int M, int K, int N, int group, void *ws, cudaStream_t s)
 {
@@ -234,6 +258,10 @@ tman_status launch_mpgemm_ternary_i8(const void *packed, const int8_t *a8, const
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
     const cuuint32_t estr[3] = {1, 1, 1};
+    // 256-channel tiles when they still give every SM two tiles or more, else 128-channel tiles
+    const long long tiles256 = (long long)((M + I8_BM - 1) / I8_BM) * ((N + 255) / 256);
+    const bool wide = tiles256 >= 2LL * sms;
+    const int bn = wide ? 256 : 128;
     CUtensorMap tmap_a;
     {
         const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
@@ -251,7 +279,7 @@ tman_status launch_mpgemm_ternary_i8(const void *packed, const int8_t *a8, const
         const cuuint64_t wt = (cuuint64_t)(K / 32);
         const cuuint64_t wdims[3] = {wt * 4, 2, (cuuint64_t)(N / 4)};
         const cuuint64_t wstrides[2] = {wt * 16, wt * 16 * 2};
-        const cuuint32_t wbox[3] = {(cuuint32_t)(I8_BK / 8), 1, (cuuint32_t)(I8_BN / 4)};
+        const cuuint32_t wbox[3] = {(cuuint32_t)(I8_BK / 8), 1, (cuuint32_t)(bn / 4)};
         if (enc(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t *>(pk + L.planes_off), wdims, wstrides,
                 wbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -265,13 +293,7 @@ tman_status launch_mpgemm_ternary_i8(const void *packed, const int8_t *a8, const
     p.status = static_cast<uint32_t *>(ws);
     p.M = M; p.K = K; p.N = N; p.group = group;
     p.tiles_m = (M + I8_BM - 1) / I8_BM;
-    p.tiles_n = (N + I8_BN - 1) / I8_BN;
-    const int tiles = p.tiles_m * p.tiles_n;
-    if (cudaFuncSetAttribute(mpgemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, I8_SMEM_BYTES) != cudaSuccess)
-        return TMAN_ERR_CUDA;
-    const int grid = tiles < sms ? tiles : sms;
-    mpgemm_i8_kernel<<<(unsigned)grid, I8_THREADS, I8_SMEM_BYTES, s>>>(tmap_a, tmap_w, p);
-    return launch_status();
+    return wide ? launch_i8<256>(tmap_a, tmap_w, p, sms, s) : launch_i8<128>(tmap_a, tmap_w, p, sms, s);
 }
 
 }  // namespace tman
