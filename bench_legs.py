@@ -75,7 +75,8 @@ def case(args, rest=()):
     import torch
     from paper_2511_11248_b200 import binding as B, helpers as H
     ap = argparse.ArgumentParser(prog="bench.py --leg case")
-    ap.add_argument("--op", choices=["gemv", "gemm"], default="gemv")
+    ap.add_argument("--op", choices=["gemv", "gemm", "ternary", "ternary_i8"], default="gemv",
+                    help="ternary: integer decode (M = 1); ternary_i8: integer prefill")
     ap.add_argument("--M", type=int, default=1)
     ap.add_argument("--K", type=int, default=4096)
     ap.add_argument("--N", type=int, default=4096)
@@ -85,12 +86,27 @@ def case(args, rest=()):
     ap.add_argument("--copies", type=int, default=1, help="rotate over this many packed copies")
     ap.add_argument("--graph", action="store_true", help="time the calls replayed from one CUDA graph")
     a = ap.parse_args(list(rest))
+    if a.op in ("ternary", "ternary_i8"):
+        a.bits = 2
     packed0, x = device_problem(torch, B, H, a.M, a.K, a.N, a.bits, a.group, seed=1)
     packed = [packed0] + [packed0.clone() for _ in range(a.copies - 1)]
-    op = B.OP_GEMV if a.op == "gemv" else B.OP_GEMM
-    fn = B.tman_mpgemv if a.op == "gemv" else B.tman_mpgemm
-    ws = workspace(torch, B, op, a.M, a.K, a.N, a.bits, a.group)
     y = torch.empty((a.M, a.N), dtype=torch.float16, device="cuda")
+    if a.op in ("ternary", "ternary_i8"):
+        # the integer path reads only the planes of the packed buffer (codes 0..3 here: timing, not parity)
+        ws = workspace(torch, B, B.OP_GEMV, 1, a.K, a.N, 2, a.group)
+        sa = torch.empty(max(a.M, 64), dtype=torch.float32, device="cuda")
+        if a.op == "ternary":
+            q = torch.empty((1, a.K), dtype=torch.int16, device="cuda")
+            B.tman_quantize_rows(x, 1, a.K, 32767, q, sa)
+            fn = lambda pk, x_, y_, M, K, N, bits, group, ws_: B.tman_mpgemv_ternary(pk, q, sa, 0.02, y_, None, 1, K, N, group, ws_)
+        else:
+            q = torch.empty((a.M, a.K), dtype=torch.int8, device="cuda")
+            B.tman_quantize_rows_i8(x, a.M, a.K, q, sa)
+            fn = lambda pk, x_, y_, M, K, N, bits, group, ws_: B.tman_mpgemm_ternary_i8(pk, q, sa, 0.02, y_, M, K, N, group, ws_)
+    else:
+        op = B.OP_GEMV if a.op == "gemv" else B.OP_GEMM
+        fn = B.tman_mpgemv if a.op == "gemv" else B.tman_mpgemm
+        ws = workspace(torch, B, op, a.M, a.K, a.N, a.bits, a.group)
     def calls():
         for i in range(a.iters):
             fn(packed[i % a.copies], x, y, a.M, a.K, a.N, a.bits, a.group, ws)

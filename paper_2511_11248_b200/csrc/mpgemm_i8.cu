@@ -15,6 +15,7 @@
 //               looks four codes at a time up in a four-entry byte table {-1, 0, +1, 0} with one byte
 //               permute; 32 INT8 per channel are stored into the K-major, 128-byte-swizzled weight tile
 //   warp 1      tcgen05.mma kind::i8 (128 x BN x 32 per instruction), commit releases the stage
+//               (two accumulator sets in tensor memory: a tile's epilogue overlaps the next tile's MMAs)
 //   last 4 warps   epilogue: tcgen05.ld of 32 tokens x 32 channels, integer -> float, the row's and the
 //               tensor's scale, fp16, 64-byte row stores
 // Every wait is bounded (about a second) and reports TMAN_ERR_TIMEOUT; tensor memory is always freed.
@@ -58,7 +59,8 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 {
     using C = I8Cfg<I8_BN>;
     constexpr int I8_STAGES = C::STAGES, I8_B_BYTES = C::B_BYTES, I8_P_PLANE_BYTES = C::P_PLANE_BYTES, I8_P_BYTES = C::P_BYTES;
-    constexpr int I8_DEQ_WARPS = C::DEQ_WARPS, I8_TMEM_COLS = I8_BN;
+    constexpr int I8_DEQ_WARPS = C::DEQ_WARPS, I8_TMEM_COLS = 2 * I8_BN;     // two accumulator sets: the epilogue of a tile
+                                                                             // overlaps the multiplications of the next
     extern __shared__ __align__(1024) uint8_t smem[];
     if (!header_matches(p.packed, p.K, p.N, 2, p.group)) {          // same answer in every CTA
         if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_BAD_PACKED);
@@ -72,9 +74,9 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     uint8_t *b_tiles = smem + I8_STAGES * I8_A_BYTES;
     uint8_t *p_tiles = smem + I8_STAGES * (I8_A_BYTES + I8_B_BYTES);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + I8_STAGES * (I8_A_BYTES + I8_B_BYTES + I8_P_BYTES));
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * I8_STAGES + 2);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * I8_STAGES + 4);
     const uint32_t loaded0 = smem_u32(bars), full0 = smem_u32(bars + I8_STAGES), empty0 = smem_u32(bars + 2 * I8_STAGES),
-                   accf = smem_u32(bars + 3 * I8_STAGES), acce = smem_u32(bars + 3 * I8_STAGES + 1);
+                   accf = smem_u32(bars + 3 * I8_STAGES), acce = smem_u32(bars + 3 * I8_STAGES + 2);   // two of each
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = p.K / I8_BK;
     const int tiles = p.tiles_m * p.tiles_n;
@@ -85,8 +87,10 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             mbar_init(full0 + 8 * s, I8_DEQ_WARPS);
             mbar_init(empty0 + 8 * s, 1);
         }
-        mbar_init(accf, 1);
-        mbar_init(acce, I8_EPI_WARPS);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(accf + 8 * b, 1);
+            mbar_init(acce + 8 * b, I8_EPI_WARPS);
+        }
         *tmem_slot = 0xFFFFFFFFu;
         fence_barrier_init();
     }
@@ -129,7 +133,8 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(I8_BN >> 3) << 17) | ((uint32_t)(I8_BM >> 4) << 24);
             uint32_t it = 0, ti = 0;
             for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
-                if (!mbar_wait(acce, (ti & 1u) ^ 1u)) { ok = false; break; }
+                const uint32_t buf = ti & 1u, acc_tmem = tmem_base + buf * (uint32_t)I8_BN;
+                if (!mbar_wait(acce + 8 * buf, ((ti >> 1) & 1u) ^ 1u)) { ok = false; break; }
                 tcgen05_fence_after();
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = (int)(it % I8_STAGES);
@@ -140,10 +145,10 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     const uint64_t bdesc = make_kmajor_sw128_desc(smem_u32(b_tiles + s * I8_B_BYTES));
 #pragma unroll
                     for (int j = 0; j < I8_BK / 32; ++j)          // 32 k = 32 bytes = two 16-byte units per instruction
-                        tcgen05_mma_i8(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc, (kb > 0 || j > 0) ? 1u : 0u);
+                        tcgen05_mma_i8(acc_tmem, adesc + 2 * j, bdesc + 2 * j, idesc, (kb > 0 || j > 0) ? 1u : 0u);
                     tcgen05_commit(empty0 + 8 * s);
                 }
-                if (ok) tcgen05_commit(accf);
+                if (ok) tcgen05_commit(accf + 8 * buf);
             }
         }
     } else if (warp < 2 + I8_DEQ_WARPS) {
@@ -172,17 +177,23 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     const uint32_t a1 = ((p0 >> 1) & 0x55555555u) | (p1 & 0xAAAAAAAAu);
                     const uint32_t X0 = a0 & 0x33333333u, X2 = (a0 >> 2) & 0x33333333u;
                     const uint32_t X1 = a1 & 0x33333333u, X3 = (a1 >> 2) & 0x33333333u;
+                    // Threads of odd strips write their two 16-byte chunks in the other order: a quarter-warp
+                    // (two strips x four words) then covers all eight chunk positions of the swizzle in
+                    // each store instruction instead of four of them twice (no bank conflicts).
+                    const bool odd = (strip & 1) != 0;
+                    const uint32_t Xa0 = odd ? X2 : X0, Xa1 = odd ? X3 : X1, Xb0 = odd ? X0 : X2, Xb1 = odd ? X1 : X3;
+                    const uint32_t ca = (uint32_t)(2 * v) + (odd ? 1u : 0u), cb = ca ^ 1u;
                     // level 2: four codes per byte permute
-                    const uint32_t o0 = __byte_perm(table, 0u, X0), o1 = __byte_perm(table, 0u, X0 >> 16);
-                    const uint32_t o2 = __byte_perm(table, 0u, X1), o3 = __byte_perm(table, 0u, X1 >> 16);
-                    const uint32_t o4 = __byte_perm(table, 0u, X2), o5 = __byte_perm(table, 0u, X2 >> 16);
-                    const uint32_t o6 = __byte_perm(table, 0u, X3), o7 = __byte_perm(table, 0u, X3 >> 16);
+                    const uint32_t o0 = __byte_perm(table, 0u, Xa0), o1 = __byte_perm(table, 0u, Xa0 >> 16);
+                    const uint32_t o2 = __byte_perm(table, 0u, Xa1), o3 = __byte_perm(table, 0u, Xa1 >> 16);
+                    const uint32_t o4 = __byte_perm(table, 0u, Xb0), o5 = __byte_perm(table, 0u, Xb0 >> 16);
+                    const uint32_t o6 = __byte_perm(table, 0u, Xb1), o7 = __byte_perm(table, 0u, Xb1 >> 16);
                     // channel row of the tile, 128 bytes per row, 16-byte chunk index XOR (row & 7)
                     const uint32_t row = (uint32_t)(4 * strip + c), xr = row & 7u;
                     const uint32_t rbase = btile + (row >> 3) * 1024u + xr * 128u;
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(rbase + (((uint32_t)(2 * v)) ^ xr) * 16u),
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(rbase + (ca ^ xr) * 16u),
                                  "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(rbase + (((uint32_t)(2 * v + 1)) ^ xr) * 16u),
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(rbase + (cb ^ xr) * 16u),
                                  "r"(o4), "r"(o5), "r"(o6), "r"(o7) : "memory");
                 }
                 fence_proxy_async_smem();
@@ -196,13 +207,14 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         uint32_t ti = 0;
         for (int t = blockIdx.x; ok && t < tiles; t += gridDim.x, ++ti) {
             const int m = tile_m0(t) + quarter * 32 + lane, n0 = tile_n0(t);
-            if (!mbar_wait(accf, ti & 1u)) { ok = false; break; }
+            const uint32_t buf = ti & 1u;
+            if (!mbar_wait(accf + 8 * buf, (ti >> 1) & 1u)) { ok = false; break; }
             tcgen05_fence_after();
             const float sc = (m < p.M) ? __ldg(p.row_scale + m) * p.w_scale : 0.f;
 #pragma unroll 1
             for (int cc = 0; cc < I8_BN / 32; ++cc) {
                 uint32_t r[32];
-                tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(32 * cc), r);
+                tcgen05_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)I8_BN + (uint32_t)(32 * cc), r);
                 tcgen05_wait_ld();
                 if (m < p.M) {
 #pragma unroll
@@ -222,7 +234,7 @@ mpgemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acce);
+            if (lane == 0) mbar_arrive(acce + 8 * buf);
         }
     }
     if (!ok && lane == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_TIMEOUT);
