@@ -329,7 +329,7 @@ mpgemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         return;
     }
     if ((smem_u32(smem) & 1023u) != 0u) {              // the swizzled tiles need 1 KB alignment (same in every CTA)
-        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_CUDA);
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)TMAN_ERR_LAYOUT);
         return;
     }
     uint8_t *a_tiles = smem;
