@@ -60,7 +60,7 @@ int tman_version(void);
 tman_status tman_packed_bytes(int K, int N, int bits, int group, size_t *out_bytes /*host*/);
 
 /* Bytes of scratch a call needs.  op: 0 = tman_mpgemv, 1 = tman_mpgemm, 2 = unpack / debug
- * extractors.  For op 0 the size depends on M: it is what the fastest plan for M rows wants;
+ * extractors and the other calls that only need the status word, 3 = tman_mpgemv_ternary.  For op 0 the size depends on M: it is what the fastest plan for M rows wants;
  * tman_mpgemv also accepts any workspace of at least the M = 1 size and then makes more passes over the
  * weights with fewer rows each (see tman_debug_gemv_plan).  The workspace must have been cleared once with tman_workspace_init before its
  * first use; calls leave it ready for the next call.  Two calls that overlap on the GPU must
@@ -158,12 +158,13 @@ tman_status tman_mpgemv_grouped(int count, const void *const *packed /*host*/, c
 tman_status tman_quantize_rows(const void *x_f16, int M, int K, int qmax, int16_t *a_i16, float *row_scale,
                                tman_stream_t stream);
 
-/* Decode of one row (M must be 1; K <= 16384): the bit-serial table lookup of tman_mpgemv on integers.
- * Tables hold exact integer sums of activations, lookups are shift-accumulated, the activation sum is
- * subtracted once (zero-point 1), K-slices are added as 32-bit integers;
- *   y[n] = fp16( row_scale[0] * w_scale * sum_k a[k] * (q[k][n] - 1) ).
- * acc_i32 (device, int32 [N], 16-byte aligned, may be NULL) receives the exact integer sums.
- * Workspace and status word as for tman_mpgemv with M = 1. */
+/* Decode of M rows (1 <= M <= 8, in passes of up to four rows; K <= 16384): the bit-serial table lookup of
+ * tman_mpgemv on integers.  Tables hold exact integer sums of activations, lookups are shift-accumulated,
+ * the activation sum is subtracted once (zero-point 1), K-slices are added as 32-bit integers;
+ *   y[m][n] = fp16( row_scale[m] * w_scale * sum_k a[m][k] * (q[k][n] - 1) ).
+ * acc_i32 (device, int32 [M][N], 16-byte aligned, may be NULL) receives the exact integer sums.
+ * Workspace: tman_workspace_bytes(3, M, K, N, 2, group), prepared with tman_workspace_init; status word
+ * as for tman_mpgemv. */
 tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const int16_t *a_i16,
                                 const float *row_scale, float w_scale, void *y_f16, int32_t *acc_i32,
                                 int M, int K, int N, int group,

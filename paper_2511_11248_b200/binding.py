@@ -18,7 +18,7 @@ STATUS_NAMES = {
     0: "TMAN_OK", 1: "TMAN_ERR_NULL", 2: "TMAN_ERR_SHAPE", 3: "TMAN_ERR_UNSUPPORTED",
     4: "TMAN_ERR_BUFFER_TOO_SMALL", 5: "TMAN_ERR_BAD_PACKED", 6: "TMAN_ERR_CUDA", 7: "TMAN_ERR_TIMEOUT",
 }
-OP_GEMV, OP_GEMM, OP_AUX = 0, 1, 2
+OP_GEMV, OP_GEMM, OP_AUX, OP_TERNARY = 0, 1, 2, 3
 
 EXPORTS = [
     "tman_status_string", "tman_version", "tman_packed_bytes", "tman_workspace_bytes",

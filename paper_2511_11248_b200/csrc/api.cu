@@ -53,6 +53,9 @@ tman_status tman_workspace_bytes(int op, int M, int K, int N, int bits, int grou
         *out_bytes = mpgemm_workspace_bytes(M, K, N);
     } else if (op == 2) {
         *out_bytes = kWsStatusBytes;
+    } else if (op == 3) {
+        if (M > 8) return TMAN_ERR_SHAPE;
+        *out_bytes = mpgemv_ternary_workspace_bytes(M, K, N);
     } else {
         return TMAN_ERR_UNSUPPORTED;
     }
@@ -165,11 +168,11 @@ tman_status tman_mpgemv_ternary(const void *packed, size_t packed_bytes, const i
     tman_status st = check_matmul(packed, packed_bytes, a_i16, y_f16, M, K, N, 2, group, workspace);
     if (st != TMAN_OK) return st;
     if (!row_scale) return TMAN_ERR_NULL;
-    if (M != 1) return TMAN_ERR_UNSUPPORTED;
+    if (M > 8) return TMAN_ERR_SHAPE;
     if (K > 16384) return TMAN_ERR_UNSUPPORTED;            // 3 * K * 32767 must stay below the "no sum pending" pattern
     if (acc_i32 && !aligned_to(acc_i32, 16)) return TMAN_ERR_SHAPE;
-    if (ws_bytes < mpgemv_workspace_bytes(1, K, N, 2)) return TMAN_ERR_BUFFER_TOO_SMALL;
-    return launch_mpgemv_ternary(packed, a_i16, row_scale, w_scale, y_f16, acc_i32, K, N, group, workspace, ws_bytes,
+    if (ws_bytes < mpgemv_ternary_workspace_bytes(M, K, N)) return TMAN_ERR_BUFFER_TOO_SMALL;
+    return launch_mpgemv_ternary(packed, a_i16, row_scale, w_scale, y_f16, acc_i32, M, K, N, group, workspace, ws_bytes,
                                  reinterpret_cast<cudaStream_t>(stream));
 }
 

@@ -128,7 +128,8 @@ struct GemvPass { int variant, rows, variant_rows, words, nkappa, ctas_per_slice
 struct GemvPlan { int npass; GemvPass pass[kGemvMaxRows]; size_t ws_bytes; double cost_us; };
 tman_status launch_quantize_rows(const void *x, int M, int K, int qmax, int16_t *a, float *s_a, cudaStream_t s);
 tman_status launch_mpgemv_ternary(const void *packed, const int16_t *a, const float *s_a, float s_w, void *y,
-                                  int32_t *acc_out, int K, int N, int group, void *ws, size_t ws_bytes, cudaStream_t s);
+                                  int32_t *acc_out, int M, int K, int N, int group, void *ws, size_t ws_bytes, cudaStream_t s);
+size_t      mpgemv_ternary_workspace_bytes(int M, int K, int N);
 tman_status launch_wait_timeout(void *ws, size_t ws_bytes, uint32_t limit, cudaStream_t s);
 GemvPlan    plan_gemv(int M, int K, int N, int bits, int sms, size_t ws_limit);
 tman_status launch_workspace_init(void *ws, size_t ws_bytes, cudaStream_t s);

@@ -233,7 +233,7 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     static_assert(!HALF || MT == 1, "half slices are for single-row tables");
-    static_assert(!INT || (HALF && !HR && !GROUPED && BITS == 2), "the integer path is built for one row of ternary weights");
+    static_assert(!INT || (!HR && !GROUPED && BITS == 2), "the integer path is built for ternary weights, fp32-held integer tables");
     static_assert(!HR || !HALF, "fp16 row pairs use whole-warp or sub-warp slices");
     constexpr int R = HR ? 2 * MT : MT;    // activation rows of this launch
     constexpr int W = HALF ? 16 : 32 / MT; // plane words (lanes) per K-slice
@@ -460,7 +460,10 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
 #pragma unroll
         for (int c = 0; c < 4; ++c) xraw[c] = make_uint4(0u, 0u, 0u, 0u);
         if (live) {
-            const uint4 *px = reinterpret_cast<const uint4 *>(p.x + (size_t)mb * p.K + (size_t)(word0 + vb) * 32);
+            // 16-bit activations either way: fp16, or the integer path's quantized values
+            const void *row = INT ? static_cast<const void *>(p.xi + (size_t)mb * p.K + (size_t)(word0 + vb) * 32)
+                                  : static_cast<const void *>(p.x + (size_t)mb * p.K + (size_t)(word0 + vb) * 32);
+            const uint4 *px = reinterpret_cast<const uint4 *>(row);
 #pragma unroll
             for (int c = 0; c < 4; ++c) xraw[c] = __ldg(px + c);
         }
@@ -478,9 +481,15 @@ __global__ void __launch_bounds__(kGemvThreads, 1) mpgemv_kernel(const GemvParam
                 float xv[8];
 #pragma unroll
                 for (int qq = 0; qq < 4; ++qq) {
-                    const float2 f = __half22float2(reinterpret_cast<const __half2 *>(&xraw[qq])[c]);
-                    xv[qq] = f.x;
-                    xv[qq + 4] = f.y;
+                    if constexpr (INT) {
+                        const short2 q2 = reinterpret_cast<const short2 *>(&xraw[qq])[c];
+                        xv[qq] = (float)q2.x;
+                        xv[qq + 4] = (float)q2.y;
+                    } else {
+                        const float2 f = __half22float2(reinterpret_cast<const __half2 *>(&xraw[qq])[c]);
+                        xv[qq] = f.x;
+                        xv[qq + 4] = f.y;
+                    }
                 }
                 float lo[16];
                 lut16(xv[0], xv[1], xv[2], xv[3], lo);
@@ -1083,15 +1092,30 @@ tman_status launch_quantize_rows_i8(const void *x, int M, int K, int8_t *a, floa
     return launch_status();
 }
 
-// One row of 16-bit integer activations times ternary weights packed as 2-bit codes (zero-point 1; the
-// packed buffer's scales and zero-points are not read).  y = fp16(s_a * s_w * sum), acc_out (may be NULL)
-// receives the exact integer sums.
+// Rows of 16-bit integer activations times ternary weights packed as 2-bit codes (zero-point 1; the
+// packed buffer's scales and zero-points are not read).  y = fp16(s_a[m] * s_w * sum), acc_out (may be NULL)
+// receives the exact integer sums.  Integer table entries are held exactly in fp32, one per row: passes of
+// one row (K-slices of 16 plane words), two rows (16 words) or four rows (8 words) per table entry.
+static void ternary_variant(int rows, int *mt, int *words)
+{
+    if (rows <= 1) { *mt = 1; *words = 16; }
+    else if (rows == 2) { *mt = 2; *words = 16; }
+    else { *mt = 4; *words = 8; }
+}
+
+size_t mpgemv_ternary_workspace_bytes(int M, int K, int N)
+{
+    int mt = 1, words = 16;
+    ternary_variant(M < 4 ? M : 4, &mt, &words);
+    const size_t nkappa = (size_t)(K / 32 + words - 1) / (size_t)words;
+    return kWsStatusBytes + nkappa * (size_t)mt * (size_t)N * sizeof(float);
+}
+
 tman_status launch_mpgemv_ternary(const void *packed, const int16_t *a, const float *s_a, float s_w, void *y,
-                                  int32_t *acc_out, int K, int N, int group, void *ws, size_t, cudaStream_t s)
+                                  int32_t *acc_out, int M, int K, int N, int group, void *ws, size_t, cudaStream_t s)
 {
     const int sms = sm_count();
     if (sms <= 0) return TMAN_ERR_CUDA;
-    if (!variant_feasible(kGemvVariants[0], K, N, sms, (size_t)-1)) return TMAN_ERR_UNSUPPORTED;
     uint8_t *w8 = static_cast<uint8_t *>(ws);
     GemvParams p = {};
     p.count = 1;
@@ -1104,21 +1128,33 @@ tman_status launch_mpgemv_ternary(const void *packed, const int16_t *a, const fl
         p.zeros[g] = reinterpret_cast<const uint16_t *>(pk + L.zeros_off);
         p.Ng[g] = g == 0 ? N : 0;
         p.col0[g] = g == 0 ? 0 : N;
-        p.y[g] = static_cast<__half *>(y);
     }
     p.N = N;
     p.x = nullptr;
-    p.xi = a;
-    p.row_scale = s_a;
     p.w_scale = s_w;
-    p.acc_out = acc_out;
     p.status = reinterpret_cast<uint32_t *>(w8);
     p.partials = reinterpret_cast<float *>(w8 + kWsStatusBytes);
-    p.K = K; p.bits = 2; p.group = group; p.M = 1;
+    p.K = K; p.bits = 2; p.group = group;
     p.group_shift = (group == 32) ? 5 : (group == 64) ? 6 : 7;
     p.nblk = K / group;
-    if (group >= 64) return launch_one<2, 1, 4, 1, 1, 0, 1, 0, 1>(p, sms, s);
-    return launch_one<2, 1, 4, 0, 1, 0, 1, 0, 1>(p, sms, s);
+    const bool pre = group >= 64;
+    for (int m0 = 0; m0 < M; m0 += 4) {
+        const int rows = (M - m0 < 4) ? (M - m0) : 4;
+        int mt = 1, words = 16;
+        ternary_variant(rows, &mt, &words);
+        if ((K / 32 + words - 1) / words > sms) return TMAN_ERR_UNSUPPORTED;      // every K-slice needs a resident CTA
+        p.M = rows;
+        p.xi = a + (size_t)m0 * K;
+        p.row_scale = s_a + m0;
+        p.acc_out = acc_out ? acc_out + (size_t)m0 * N : nullptr;
+        for (int g = 0; g < kGemvMaxGroup; ++g) p.y[g] = static_cast<__half *>(y) + (size_t)m0 * N;
+        tman_status st;
+        if (mt == 1) st = pre ? launch_one<2, 1, 4, 1, 1, 0, 1, 0, 1>(p, sms, s) : launch_one<2, 1, 4, 0, 1, 0, 1, 0, 1>(p, sms, s);
+        else if (mt == 2) st = pre ? launch_one<2, 2, 2, 1, 0, 0, 1, 0, 1>(p, sms, s) : launch_one<2, 2, 2, 0, 0, 0, 1, 0, 1>(p, sms, s);
+        else st = pre ? launch_one<2, 4, 1, 1, 0, 0, 1, 0, 1>(p, sms, s) : launch_one<2, 4, 1, 0, 0, 0, 1, 0, 1>(p, sms, s);
+        if (st != TMAN_OK) return st;
+    }
+    return TMAN_OK;
 }
 
 tman_status launch_mpgemv(const void *packed, const void *x, void *y, int M, int K, int N, int bits,

@@ -61,7 +61,7 @@ def test_ternary_decode_matches_the_integer_oracle(K, N, group):
     a = H.guarded_bytes(K * 2, "a_i16").view(torch.int16).view(1, K)
     s = H.guarded_bytes(256, "row_scale").view(torch.float32)
     B.tman_quantize_rows(xd, 1, K, 32767, a, s)
-    ws = H.alloc_workspace(B.OP_GEMV, 1, K, N, 2, group)
+    ws = H.alloc_workspace(B.OP_TERNARY, 1, K, N, 2, group)
     y = H.alloc_y(1, N)
     acc = H.guarded_bytes(N * 4, "acc_i32").view(torch.int32).view(1, N)
     acc.fill_(-12345)
@@ -96,9 +96,9 @@ def test_ternary_closed_forms_and_refusals():
         B.tman_mpgemv_ternary(packed, a, s, s_w, y, acc, 1, K, N, 64, ws)
         assert B.tman_read_status(ws) == 0
         assert bool((acc == want).all())
-    with pytest.raises(B.TmanError) as e:                      # one row only
-        B.tman_mpgemv_ternary(packed, a, s, s_w, y, acc, 2, K, N, 64, ws)
-    assert e.value.status == 3
+    with pytest.raises(B.TmanError) as e:                      # at most eight rows
+        B.tman_mpgemv_ternary(packed, a, s, s_w, y, acc, 9, K, N, 64, ws)
+    assert e.value.status == 2
     junk = torch.zeros_like(packed)
     y.fill_(3.0)
     B.tman_mpgemv_ternary(junk, a, s, s_w, y, acc, 1, K, N, 64, ws)
@@ -159,3 +159,27 @@ def test_int8_prefill_matches_the_integer_oracle(M, K, N, group):
     y.fill_(3.0)
     B.tman_mpgemm_ternary_i8(torch.zeros_like(packed), a8, s, s_w, y, M, K, N, group, ws)
     assert B.tman_read_status(ws) == 5 and bool((y == 3.0).all())
+
+
+@pytest.mark.parametrize("M,K,N,group", [(2, 1024, 40, 64), (3, 2560, 264, 128), (4, 6912, 2560, 128), (5, 1152, 72, 32),
+                                         (8, 2560, 6912, 64), (7, 16384, 16, 128)])
+def test_ternary_decode_with_several_rows(M, K, N, group):
+    x, t, q, s_w = ternary_case(M, K, N, seed=7 * M + K + N, spread=1.5)
+    a_ref, s_ref = oi.quantize_rows(x, 32767)
+    acc_ref = oi.ternary_lut_matmul(a_ref, q)
+    y_ref = oi.scale_result(acc_ref, s_ref, float(np.float32(s_w)))
+    packed = pack_ternary(q, group)
+    xd = torch.from_numpy(x.view(np.int16)).cuda().view(torch.float16)
+    a = H.guarded_bytes(M * K * 2, "a_i16").view(torch.int16).view(M, K)
+    s = H.guarded_bytes(256, "row_scale").view(torch.float32)
+    B.tman_quantize_rows(xd, M, K, 32767, a, s)
+    ws = H.guarded_bytes(B.tman_workspace_bytes(B.OP_TERNARY, M, K, N, 2, group), "workspace")
+    B.tman_workspace_init(ws)
+    y = H.alloc_y(M, N)
+    acc = H.guarded_bytes(M * N * 4, "acc_i32").view(torch.int32).view(M, N)
+    for _ in range(2):
+        B.tman_mpgemv_ternary(packed, a, s, s_w, y, acc, M, K, N, group, ws)
+        assert B.tman_read_status(ws) == 0
+        H.check_guards()
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+        assert np.all(np.abs(H.to_f64(y) - y_ref) <= np.abs(y_ref) * 2.0 ** -10 + 1e-7)
