@@ -260,7 +260,8 @@ tman_status tman_debug_luts(const void *x_f16, int M, int K, float *lut, tman_st
  *           3  Sequential: the product's dequantization with a ring of one stage, so that the load, the
  *              dequantization and the multiplication of a k-block follow one another
  *   wt_f16  used by variant 2 only (else may be NULL).
- * Variants 1-3 exist for bits == 4 (TMAN_ERR_UNSUPPORTED otherwise). */
+ * Variants 1-3 exist for bits == 4 (TMAN_ERR_UNSUPPORTED otherwise); variant 2 additionally wants N to be a
+ * multiple of 32 (TMAN_ERR_UNSUPPORTED otherwise). */
 tman_status tman_debug_mpgemm_variant(int variant, const void *packed, size_t packed_bytes, const void *x_f16,
                                       void *y_f16, int M, int K, int N, int bits, int group, const void *wt_f16,
                                       void *workspace, size_t ws_bytes, tman_stream_t stream);

@@ -1071,6 +1071,7 @@ tman_status launch_mpgemm_variant(int variant, const void *packed, const void *x
     if (variant < kGemmProduct || variant > kGemmSequential) return TMAN_ERR_UNSUPPORTED;
     if (variant != kGemmProduct && bits != 4) return TMAN_ERR_UNSUPPORTED;
     if (variant == kGemmLoadFull && (!wt_f16 || (reinterpret_cast<uintptr_t>(wt_f16) & 15) != 0)) return TMAN_ERR_SHAPE;
+    if (variant == kGemmLoadFull && (N % 32) != 0) return TMAN_ERR_UNSUPPORTED;     // whole 32-channel units only
     if ((reinterpret_cast<uintptr_t>(x) & 15) != 0 || (reinterpret_cast<uintptr_t>(y) & 15) != 0) return TMAN_ERR_SHAPE;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return TMAN_ERR_CUDA;
